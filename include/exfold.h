@@ -1,0 +1,187 @@
+/*
+ * exfold.h - C ABI of the B200 (sm_100a) folded Mixture-of-Experts layer (ExFold).
+ *
+ * One MoE layer with N routed SwiGLU experts (+ an optional always-on shared expert):
+ *     E_e(x) = W_down^(e) ( silu(W_gate^(e) x) * (W_up^(e) x) )                 (Eq. 1)
+ *     S_K(x) = Top-K router logits, a_e = softmax restricted to S_K              (Eq. 2)
+ *     MoE(x) = sum_{e in S_K} a_e E_e(x)  (+ shared expert, weight 1)            (Eq. 3)
+ * Folding executes only a retained subset of the routed experts and moves the gate
+ * weight of every excluded expert s onto its minimum-loss retained expert t, scaled by
+ * the calibrated pairwise scalar S[s][t] (Eq. 4, 12). Two modes:
+ *     prefill: per token, keep the K' routes with the largest a_e h_e   (Eq. 10, 13)
+ *     decode : per batch, keep a pool of at most M experts ranked by
+ *              sum_i a_{i,e} h_e, remap every other route in place       (Eq. 11, 14)
+ *
+ * Conventions for every call
+ *   - All tensors are dense, row-major. Weights are stored like nn.Linear (out x in):
+ *     W_gate, W_up [N+n_shared][I][d], W_down [N+n_shared][d][I]; the shared expert, if
+ *     any, is expert index N. x, W_*, y have the layer dtype; router logits and all
+ *     tables are fp32; indices are int32.
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the
+ *     caller. The library allocates no device memory and keeps no state between calls:
+ *     all scratch lives in the caller's workspace `ws` (exfold_workspace_bytes; 256-byte
+ *     aligned). Calls that share a workspace must be ordered on one stream.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
+ *     default stream) and return without synchronising, except exfold_device_status.
+ *   - Return value: EXFOLD_OK (0), a negative error (nothing was launched), or a positive
+ *     warning. Arguments are validated on the host before anything is launched.
+ *   - Every wait inside a kernel is bounded; a kernel that gives up records
+ *     EXFOLD_ERR_DEVICE_TIMEOUT in the workspace's status word and returns.
+ *   - bf16 layers need d and I to be multiples of 64; N <= 256, K <= 32.
+ */
+#ifndef EXFOLD_H_
+#define EXFOLD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { EXFOLD_F32 = 0, EXFOLD_BF16 = 1 } exfold_dtype;
+
+enum {
+    EXFOLD_OK = 0,
+    EXFOLD_ERR_INVALID_ARG = -1,
+    EXFOLD_ERR_UNSUPPORTED = -2,
+    EXFOLD_ERR_WORKSPACE_TOO_SMALL = -3,
+    EXFOLD_ERR_CUDA = -4,
+    EXFOLD_ERR_DEVICE_TIMEOUT = -5,
+    EXFOLD_WARN_UNOBSERVED_EXPERT = 1
+};
+
+/* Shape of the layer (Eq. 1-3). */
+typedef struct {
+    int32_t n_experts; /* N routed experts, 2..256 */
+    int32_t n_shared;  /* 0 or 1 shared expert, stored as expert N */
+    int32_t hidden;    /* d */
+    int32_t inter;     /* I */
+    int32_t top_k;     /* K of the original router, 1..32, <= N */
+    int32_t dtype;     /* exfold_dtype of x, W_*, y */
+} exfold_layer;
+
+/*
+ * Calibration tables of one layer (device, caller-owned, fp32).
+ *   S [N][N]  scalar projector, row = source expert, column = target expert (Eq. 8)
+ *   L [N][N]  projection loss (Eq. 9)
+ *   h [N]     output-norm estimate of each expert; lnh[e] = (float)log((double)h[e])
+ *   n_obs [N][N] number of calibration tokens seen per pair (written by calibrate; may be NULL)
+ */
+typedef struct {
+    float *S;
+    float *L;
+    float *h;
+    float *lnh;
+    int32_t *n_obs;
+} exfold_tables;
+
+/* Options of exfold_calibrate ("Calibration protocol": lambda = 1e-3, clip [-4,4]). */
+typedef struct {
+    float lambda;  /* ridge term of Eq. 8 */
+    float clip_lo; /* scalars are clipped to [clip_lo, clip_hi] before the loss is taken */
+    float clip_hi;
+    float eps;     /* added to the denominator of the normalised loss (appendix form of Eq. 9) */
+    int32_t mode;  /* 0: pairs observed when both experts are in a token's Top-K; 1: every expert sees every token */
+} exfold_calib_opts;
+
+/* Optional routing metadata written by exfold_moe_prefill (device pointers; any may be NULL). */
+typedef struct {
+    int32_t *ids;      /* [T][K']   retained experts, descending a_e h_e            */
+    float *w;          /* [T][K']   folded weights (Eq. 13)                         */
+    int32_t *omit_src; /* [T][K-K'] omitted experts, descending a_e h_e             */
+    int32_t *omit_tgt; /* [T][K-K'] their minimum-loss targets (Eq. 12)             */
+    int32_t *perm;     /* [T*K']    route indices i*K'+j sorted by (expert, i, j)   */
+    int32_t *offsets;  /* [N+1]     first sorted position of each expert            */
+} exfold_prefill_meta;
+
+/* Optional routing metadata written by exfold_moe_decode (device pointers; any may be NULL). */
+typedef struct {
+    int32_t *pool_ids;   /* [M]  pool experts, descending score, -1 padded (Eq. 11)        */
+    int32_t *pool_size;  /* [1]  min(M, size of the batch's expert union)                  */
+    uint32_t *pool_mask; /* [ceil(N/32)] bit e set when expert e is in the pool            */
+    int32_t *ids;        /* [B][K] remapped expert of every routed slot (Eq. 14)           */
+    float *w;            /* [B][K] remapped weight of every routed slot                    */
+    int32_t *target;     /* [N]  target[s]: s itself if in the pool, else its min-loss pool expert */
+    float *scale;        /* [N]  1 or S[s][target[s]]                                      */
+} exfold_decode_meta;
+
+/*
+ * Bytes of workspace needed by any call on `layer` with up to max_tokens tokens
+ * (T, B or calibration tokens) and up to routes_per_token executed routes per token
+ * (K' for prefill, K for decode and calibration). Returns 0 for an invalid layer.
+ */
+size_t exfold_workspace_bytes(const exfold_layer *layer, int64_t max_tokens, int32_t routes_per_token);
+
+/*
+ * Offline calibration of the pairwise scalar projector (Eq. 6-9 and the appendix's
+ * shared-scalar and normalised-loss forms). Runs the routed experts on m calibration
+ * tokens x_cal [m][d] with logits_cal [m][N], accumulates per ordered pair (s,t) the
+ * sums of w<v,u>, w|v|^2, w|u|^2 with w = |u| (u = E_s(x), v = E_t(x)) in double, and
+ * writes S, L, h, lnh (and n_obs if non-NULL) into `out`. S_ee = 1, L_ee = 0; a pair
+ * never observed gets S = 0, L = 1e30; an expert never observed gets the mean h of the
+ * others and the call returns EXFOLD_WARN_UNOBSERVED_EXPERT after synchronising the
+ * stream (this call is off the serving path and does synchronise).
+ */
+int exfold_calibrate(const exfold_layer *layer, const void *x_cal, const float *logits_cal, int64_t m,
+                     const void *w_gate, const void *w_up, const void *w_down,
+                     const exfold_calib_opts *opts, exfold_tables *out, void *ws, size_t ws_bytes,
+                     void *cuda_stream);
+
+/*
+ * Prefill: token-level Top-K folding (Eq. 10, 12, 13, then Eq. 1 and 4 over the retained
+ * routes only). x [T][d], logits [T][N] -> y [T][d]. k_pre = K' in [1, K]; k_pre = K is the
+ * unfolded layer. Each token executes exactly K' routed experts (+ the shared expert).
+ * Ranking uses key = logit + lnh[e] (one fp32 add; same order as a_e h_e).
+ */
+int exfold_moe_prefill(const exfold_layer *layer, const void *x, const float *logits, int64_t T,
+                       const void *w_gate, const void *w_up, const void *w_down,
+                       const exfold_tables *tables, int32_t k_pre, void *y,
+                       const exfold_prefill_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Decode: batch-level expert-pool folding (Eq. 11, 12, 14, then Eq. 1 and 4 over the pool
+ * only). x [B][d], logits [B][N] -> y [B][d], B <= 256. pool_m = M in [1, N]; the pool is
+ * the whole expert union of the batch when that has at most M experts, so pool_m = N is the
+ * unfolded layer. Scores are accumulated in double, tokens ascending. Only the pool's (and
+ * the shared expert's) weights are read.
+ */
+int exfold_moe_decode(const exfold_layer *layer, const void *x, const float *logits, int64_t B,
+                      const void *w_gate, const void *w_up, const void *w_down,
+                      const exfold_tables *tables, int32_t pool_m, void *y,
+                      const exfold_decode_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * The same two calls for activations that live in HOST memory (pinned for real overlap):
+ * x_host, logits_host and y_host are host pointers; the call stages them through the
+ * workspace with asynchronous copies on the stream (x and logits in before the layer, y out
+ * after it). Weights, tables, metadata and workspace stay device pointers. The workspace
+ * must be exfold_workspace_bytes(...) + exfold_host_staging_bytes(...) large.
+ */
+size_t exfold_host_staging_bytes(const exfold_layer *layer, int64_t max_tokens);
+int exfold_moe_prefill_host(const exfold_layer *layer, const void *x_host, const float *logits_host,
+                            int64_t T, const void *w_gate, const void *w_up, const void *w_down,
+                            const exfold_tables *tables, int32_t k_pre, void *y_host,
+                            const exfold_prefill_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
+int exfold_moe_decode_host(const exfold_layer *layer, const void *x_host, const float *logits_host,
+                           int64_t B, const void *w_gate, const void *w_up, const void *w_down,
+                           const exfold_tables *tables, int32_t pool_m, void *y_host,
+                           const exfold_decode_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Synchronises the stream and decodes the status word the kernels keep at the start of the
+ * workspace: EXFOLD_OK, EXFOLD_ERR_DEVICE_TIMEOUT (a bounded wait ran out), or
+ * EXFOLD_ERR_CUDA. Clears the word. The only synchronising call on the serving path.
+ */
+int exfold_device_status(void *ws, void *cuda_stream);
+
+/* Human-readable name of a status code (static storage). */
+const char *exfold_status_string(int status);
+
+/* Number of kernels of this library launched by this process so far (for launch accounting). */
+int64_t exfold_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EXFOLD_H_ */

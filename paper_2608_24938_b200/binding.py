@@ -1,0 +1,212 @@
+"""ctypes binding of libexfold.so: argument marshalling only.
+
+Every function has the name and the arguments of its C counterpart in include/exfold.h;
+tensors are torch tensors whose data pointers are passed through. All computation happens
+in the CUDA library; there is no fallback: if the library is missing, importing fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libexfold.so")
+
+EXFOLD_F32, EXFOLD_BF16 = 0, 1
+EXFOLD_OK = 0
+EXFOLD_ERR_INVALID_ARG = -1
+EXFOLD_ERR_UNSUPPORTED = -2
+EXFOLD_ERR_WORKSPACE_TOO_SMALL = -3
+EXFOLD_ERR_CUDA = -4
+EXFOLD_ERR_DEVICE_TIMEOUT = -5
+EXFOLD_WARN_UNOBSERVED_EXPERT = 1
+
+EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibrate", "exfold_moe_prefill",
+           "exfold_moe_decode", "exfold_moe_prefill_host", "exfold_moe_decode_host", "exfold_device_status",
+           "exfold_status_string", "exfold_launch_count"]
+
+
+class exfold_layer(C.Structure):
+    _fields_ = [("n_experts", C.c_int32), ("n_shared", C.c_int32), ("hidden", C.c_int32), ("inter", C.c_int32),
+                ("top_k", C.c_int32), ("dtype", C.c_int32)]
+
+
+class exfold_tables(C.Structure):
+    _fields_ = [("S", C.c_void_p), ("L", C.c_void_p), ("h", C.c_void_p), ("lnh", C.c_void_p), ("n_obs", C.c_void_p)]
+
+
+class exfold_calib_opts(C.Structure):
+    _fields_ = [("lambda_", C.c_float), ("clip_lo", C.c_float), ("clip_hi", C.c_float), ("eps", C.c_float),
+                ("mode", C.c_int32)]
+
+
+class exfold_prefill_meta(C.Structure):
+    _fields_ = [("ids", C.c_void_p), ("w", C.c_void_p), ("omit_src", C.c_void_p), ("omit_tgt", C.c_void_p),
+                ("perm", C.c_void_p), ("offsets", C.c_void_p)]
+
+
+class exfold_decode_meta(C.Structure):
+    _fields_ = [("pool_ids", C.c_void_p), ("pool_size", C.c_void_p), ("pool_mask", C.c_void_p), ("ids", C.c_void_p),
+                ("w", C.c_void_p), ("target", C.c_void_p), ("scale", C.c_void_p)]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2608_24938_b200.build` "
+                          "(there is no CPU or PyTorch fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i64, i32, sz = C.c_void_p, C.c_int64, C.c_int32, C.c_size_t
+    lib.exfold_workspace_bytes.restype = sz
+    lib.exfold_workspace_bytes.argtypes = [C.POINTER(exfold_layer), i64, i32]
+    lib.exfold_host_staging_bytes.restype = sz
+    lib.exfold_host_staging_bytes.argtypes = [C.POINTER(exfold_layer), i64]
+    lib.exfold_calibrate.restype = C.c_int
+    lib.exfold_calibrate.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_calib_opts),
+                                     C.POINTER(exfold_tables), vp, sz, vp]
+    for fn in (lib.exfold_moe_prefill, lib.exfold_moe_prefill_host):
+        fn.restype = C.c_int
+        fn.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables), i32, vp,
+                       C.POINTER(exfold_prefill_meta), vp, sz, vp]
+    for fn in (lib.exfold_moe_decode, lib.exfold_moe_decode_host):
+        fn.restype = C.c_int
+        fn.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables), i32, vp,
+                       C.POINTER(exfold_decode_meta), vp, sz, vp]
+    lib.exfold_device_status.restype = C.c_int
+    lib.exfold_device_status.argtypes = [vp, vp]
+    lib.exfold_status_string.restype = C.c_char_p
+    lib.exfold_status_string.argtypes = [C.c_int]
+    lib.exfold_launch_count.restype = i64
+    lib.exfold_launch_count.argtypes = []
+    return lib
+
+
+lib = _load()
+
+
+class ExfoldError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {exfold_status_string(code)} ({code})")
+        self.code = code
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors passed to the library must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def make_layer(n_experts: int, n_shared: int, hidden: int, inter: int, top_k: int, dtype) -> exfold_layer:
+    if isinstance(dtype, torch.dtype):
+        dtype = {torch.float32: EXFOLD_F32, torch.bfloat16: EXFOLD_BF16}[dtype]
+    elif isinstance(dtype, str):
+        dtype = {"f32": EXFOLD_F32, "bf16": EXFOLD_BF16}[dtype]
+    return exfold_layer(n_experts, n_shared, hidden, inter, top_k, dtype)
+
+
+def make_tables(S, L, h, lnh, n_obs=None) -> exfold_tables:
+    for t in (S, L, h, lnh):
+        assert t.dtype == torch.float32
+    return exfold_tables(_ptr(S), _ptr(L), _ptr(h), _ptr(lnh), _ptr(n_obs))
+
+
+def exfold_status_string(code: int) -> str:
+    return lib.exfold_status_string(code).decode()
+
+
+def exfold_launch_count() -> int:
+    return int(lib.exfold_launch_count())
+
+
+def exfold_workspace_bytes(layer: exfold_layer, max_tokens: int, routes_per_token: int) -> int:
+    return int(lib.exfold_workspace_bytes(C.byref(layer), max_tokens, routes_per_token))
+
+
+def exfold_host_staging_bytes(layer: exfold_layer, max_tokens: int) -> int:
+    return int(lib.exfold_host_staging_bytes(C.byref(layer), max_tokens))
+
+
+def alloc_workspace(layer: exfold_layer, max_tokens: int, routes_per_token: int, device="cuda",
+                    host_staging: bool = False) -> torch.Tensor:
+    n = exfold_workspace_bytes(layer, max_tokens, routes_per_token)
+    if n == 0:
+        raise ExfoldError(EXFOLD_ERR_INVALID_ARG, "exfold_workspace_bytes")
+    if host_staging:
+        n += exfold_host_staging_bytes(layer, max_tokens)
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def exfold_device_status(ws: torch.Tensor, stream=None) -> int:
+    return int(lib.exfold_device_status(_ptr(ws), _stream(stream)))
+
+
+def exfold_calibrate(layer, x_cal, logits_cal, w_gate, w_up, w_down, out: exfold_tables, ws, lam=1e-3,
+                     clip_lo=-4.0, clip_hi=4.0, eps=1e-12, mode=0, stream=None) -> int:
+    opts = exfold_calib_opts(lam, clip_lo, clip_hi, eps, mode)
+    rc = lib.exfold_calibrate(C.byref(layer), _ptr(x_cal), _ptr(logits_cal), x_cal.shape[0], _ptr(w_gate),
+                              _ptr(w_up), _ptr(w_down), C.byref(opts), C.byref(out), _ptr(ws), ws.numel(),
+                              _stream(stream))
+    if rc < 0:
+        raise ExfoldError(rc, "exfold_calibrate")
+    return rc
+
+
+def _prefill_meta(meta: Optional[dict]):
+    if not meta:
+        return None
+    return C.byref(exfold_prefill_meta(*[_ptr(meta.get(k)) for k in
+                                         ("ids", "w", "omit_src", "omit_tgt", "perm", "offsets")]))
+
+
+def _decode_meta(meta: Optional[dict]):
+    if not meta:
+        return None
+    return C.byref(exfold_decode_meta(*[_ptr(meta.get(k)) for k in
+                                        ("pool_ids", "pool_size", "pool_mask", "ids", "w", "target", "scale")]))
+
+
+def exfold_moe_prefill(layer, x, logits, w_gate, w_up, w_down, tables: exfold_tables, k_pre: int, y, ws,
+                       meta: Optional[dict] = None, stream=None, check: bool = True) -> int:
+    rc = lib.exfold_moe_prefill(C.byref(layer), _ptr(x), _ptr(logits), x.shape[0], _ptr(w_gate), _ptr(w_up),
+                                _ptr(w_down), C.byref(tables), k_pre, _ptr(y), _prefill_meta(meta), _ptr(ws),
+                                ws.numel(), _stream(stream))
+    if check and rc != 0:
+        raise ExfoldError(rc, "exfold_moe_prefill")
+    return rc
+
+
+def exfold_moe_decode(layer, x, logits, w_gate, w_up, w_down, tables: exfold_tables, pool_m: int, y, ws,
+                      meta: Optional[dict] = None, stream=None, check: bool = True) -> int:
+    rc = lib.exfold_moe_decode(C.byref(layer), _ptr(x), _ptr(logits), x.shape[0], _ptr(w_gate), _ptr(w_up),
+                               _ptr(w_down), C.byref(tables), pool_m, _ptr(y), _decode_meta(meta), _ptr(ws),
+                               ws.numel(), _stream(stream))
+    if check and rc != 0:
+        raise ExfoldError(rc, "exfold_moe_decode")
+    return rc
+
+
+def exfold_moe_prefill_host(layer, x_host, logits_host, w_gate, w_up, w_down, tables, k_pre, y_host, ws,
+                            meta=None, stream=None, check: bool = True) -> int:
+    rc = lib.exfold_moe_prefill_host(C.byref(layer), _ptr(x_host), _ptr(logits_host), x_host.shape[0], _ptr(w_gate),
+                                     _ptr(w_up), _ptr(w_down), C.byref(tables), k_pre, _ptr(y_host),
+                                     _prefill_meta(meta), _ptr(ws), ws.numel(), _stream(stream))
+    if check and rc != 0:
+        raise ExfoldError(rc, "exfold_moe_prefill_host")
+    return rc
+
+
+def exfold_moe_decode_host(layer, x_host, logits_host, w_gate, w_up, w_down, tables, pool_m, y_host, ws,
+                           meta=None, stream=None, check: bool = True) -> int:
+    rc = lib.exfold_moe_decode_host(C.byref(layer), _ptr(x_host), _ptr(logits_host), x_host.shape[0], _ptr(w_gate),
+                                    _ptr(w_up), _ptr(w_down), C.byref(tables), pool_m, _ptr(y_host),
+                                    _decode_meta(meta), _ptr(ws), ws.numel(), _stream(stream))
+    if check and rc != 0:
+        raise ExfoldError(rc, "exfold_moe_decode_host")
+    return rc

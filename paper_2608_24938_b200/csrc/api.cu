@@ -1,0 +1,472 @@
+// C ABI of the folded-MoE library: argument validation, workspace planning, TMA tensor maps
+// and the launch sequences of the three calls. No device memory is allocated here.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace exfold {
+
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+namespace {
+
+// ------------------------------------------------------------------ workspace plan
+struct Plan {
+    size_t status, ids, w, omit_src, omit_tgt, block_hist, offsets, work_start, totals, perm, row_tok, row_w,
+        row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
+        xs, H, y32, out, total;
+};
+
+bool valid_layer(const exfold_layer* l) {
+    if (!l) return false;
+    if (l->n_experts < 2 || l->n_experts > kMaxExperts) return false;
+    if (l->n_shared < 0 || l->n_shared > 1) return false;
+    if (l->top_k < 1 || l->top_k > kMaxTopK || l->top_k > l->n_experts) return false;
+    if (l->hidden < 1 || l->inter < 1) return false;
+    if (l->dtype != EXFOLD_F32 && l->dtype != EXFOLD_BF16) return false;
+    if (l->dtype == EXFOLD_BF16 && (l->hidden % 64 != 0 || l->inter % 64 != 0)) return false;
+    if (l->dtype == EXFOLD_F32 && (l->hidden % 4 != 0)) return false;
+    return true;
+}
+
+Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
+    Plan p{};
+    const int N = l.n_experts, G = N + l.n_shared;
+    const size_t Rm = (size_t)Tm * Kr, Rtot = Rm + (size_t)Tm * l.n_shared;
+    const size_t nblk = (size_t)(Tm + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = off;
+        off = align_up(off + bytes, 256);
+        return at;
+    };
+    p.status = take(sizeof(DeviceStatus));
+    p.ids = take(Rm * 4);
+    p.w = take(Rm * 4);
+    p.omit_src = take((size_t)Tm * l.top_k * 4);
+    p.omit_tgt = take((size_t)Tm * l.top_k * 4);
+    p.block_hist = take(nblk * N * 4);
+    p.offsets = take((G + 2) * 4);
+    p.work_start = take((G + 2) * 4);
+    p.totals = take(16);
+    p.perm = take(Rm * 4);
+    p.row_tok = take(Rtot * 4);
+    p.row_w = take(Rtot * 4);
+    p.row_exp = take(Rtot * 4);
+    p.pool_ids = take((size_t)N * 4);
+    p.pool_size = take(16);
+    p.pool_mask = take(32);
+    p.target = take((size_t)N * 4);
+    p.scale = take((size_t)N * 4);
+    p.grp_expert = take((G + 2) * 4);
+    p.grp_off = take((G + 2) * 4);
+    p.n_groups = take(16);
+    p.zeros = take((size_t)N * 4);
+    p.calib = take((size_t)N * N * (3 * 8 + 4) + (size_t)N * (8 + 4) + 256);
+    // large buffers: the bf16 pipeline (sorted rows, H, fp32 accumulator) and the SIMT path's
+    // per-route outputs are never live at the same time and share one region
+    p.big = off;
+    size_t a = 0;
+    if (l.dtype == EXFOLD_BF16) {
+        p.xs = p.big;
+        a = align_up(Rtot * (size_t)l.hidden * 2, 1024);
+        p.H = p.big + a;
+        a += align_up(Rtot * (size_t)l.inter * 2, 1024);
+        p.y32 = p.big + a;
+        a += align_up((size_t)Tm * l.hidden * 4, 1024);
+    }
+    p.out = p.big;
+    size_t b = align_up(Rtot * (size_t)l.hidden * 4, 1024);
+    p.total = p.big + (a > b ? a : b);
+    return p;
+}
+
+template <typename T>
+T* at(void* ws, size_t off) {
+    return reinterpret_cast<T*>(reinterpret_cast<char*>(ws) + off);
+}
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][cols] row-major; box = box_rows x 64 columns (128 bytes), 128-byte swizzle
+bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+#define EXFOLD_CUDA(call)                                 \
+    do {                                                  \
+        cudaError_t e__ = (call);                         \
+        if (e__ != cudaSuccess) return EXFOLD_ERR_CUDA;   \
+    } while (0)
+
+int copy_meta(void* dst, const void* src, size_t bytes, cudaStream_t s) {
+    if (dst == nullptr || bytes == 0) return EXFOLD_OK;
+    EXFOLD_CUDA(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, s));
+    return EXFOLD_OK;
+}
+
+int check_common(const exfold_layer* layer, const void* x, const float* logits, int64_t T, const void* wg,
+                 const void* wu, const void* wd, const exfold_tables* t, void* y, void* ws) {
+    if (!valid_layer(layer)) return EXFOLD_ERR_INVALID_ARG;
+    if (!x || !logits || !wg || !wu || !wd || !y || !ws) return EXFOLD_ERR_INVALID_ARG;
+    if (!t || !t->S || !t->L || !t->h || !t->lnh) return EXFOLD_ERR_INVALID_ARG;
+    if (T < 1 || T > (int64_t)1 << 24) return EXFOLD_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(wg) || !aligned16(wu) || !aligned16(wd) ||
+        (reinterpret_cast<uintptr_t>(ws) & 255) != 0)
+        return EXFOLD_ERR_INVALID_ARG;
+    return EXFOLD_OK;
+}
+
+}  // namespace
+}  // namespace exfold
+
+using namespace exfold;
+
+extern "C" {
+
+size_t exfold_workspace_bytes(const exfold_layer* layer, int64_t max_tokens, int32_t routes_per_token) {
+    if (!valid_layer(layer) || max_tokens < 1 || routes_per_token < 1 || routes_per_token > kMaxExperts) return 0;
+    return make_plan(*layer, max_tokens, routes_per_token).total;
+}
+
+size_t exfold_host_staging_bytes(const exfold_layer* layer, int64_t max_tokens) {
+    if (!valid_layer(layer) || max_tokens < 1) return 0;
+    const size_t el = layer->dtype == EXFOLD_BF16 ? 2 : 4;
+    return 2 * align_up((size_t)max_tokens * layer->hidden * el, 256) +
+           align_up((size_t)max_tokens * layer->n_experts * 4, 256);
+}
+
+int64_t exfold_launch_count(void) { return g_launches.load(); }
+
+const char* exfold_status_string(int status) {
+    switch (status) {
+        case EXFOLD_OK: return "ok";
+        case EXFOLD_ERR_INVALID_ARG: return "invalid argument";
+        case EXFOLD_ERR_UNSUPPORTED: return "unsupported configuration";
+        case EXFOLD_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case EXFOLD_ERR_CUDA: return "CUDA error";
+        case EXFOLD_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+        case EXFOLD_WARN_UNOBSERVED_EXPERT: return "warning: an expert was never observed during calibration";
+        default: return "unknown status";
+    }
+}
+
+int exfold_device_status(void* ws, void* cuda_stream) {
+    if (!ws) return EXFOLD_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return EXFOLD_ERR_CUDA;
+    int code = 0;
+    if (cudaMemcpy(&code, ws, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return EXFOLD_ERR_CUDA;
+    if (cudaMemset(ws, 0, sizeof(DeviceStatus)) != cudaSuccess) return EXFOLD_ERR_CUDA;
+    if (code == 0) return EXFOLD_OK;
+    return code == EXFOLD_ERR_DEVICE_TIMEOUT ? EXFOLD_ERR_DEVICE_TIMEOUT : EXFOLD_ERR_CUDA;
+}
+
+int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* logits, int64_t T, const void* w_gate,
+                       const void* w_up, const void* w_down, const exfold_tables* tables, int32_t k_pre, void* y,
+                       const exfold_prefill_meta* meta, void* ws, size_t ws_bytes, void* cuda_stream) {
+    int rc = check_common(layer, x, logits, T, w_gate, w_up, w_down, tables, y, ws);
+    if (rc != EXFOLD_OK) return rc;
+    const exfold_layer& l = *layer;
+    if (k_pre < 1 || k_pre > l.top_k) return EXFOLD_ERR_INVALID_ARG;
+    const int N = l.n_experts, K = l.top_k, Kp = k_pre, d = l.hidden, I = l.inter, G = N + l.n_shared;
+    const int64_t R = T * Kp, Rtot = R + T * l.n_shared;
+    if (Rtot > (int64_t)1 << 30) return EXFOLD_ERR_UNSUPPORTED;
+    const Plan pl = make_plan(l, T, Kp);
+    if (ws_bytes < pl.total) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const bool bf16 = l.dtype == EXFOLD_BF16;
+    const bool direct = bf16 && Kp == 1 && l.n_shared == 0;  // every token is written exactly once
+
+    CUtensorMap tm_xs, tm_x, tm_wg, tm_wu, tm_h, tm_wd;
+    if (bf16) {
+        const uint64_t E = (uint64_t)G;
+        bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)R, d, 128) && make_tmap(&tm_x, x, (uint64_t)T, d, 128) &&
+                  make_tmap(&tm_wg, w_gate, E * I, d, 128) && make_tmap(&tm_wu, w_up, E * I, d, 128) &&
+                  make_tmap(&tm_h, at<char>(ws, pl.H), (uint64_t)Rtot, I, 128) &&
+                  make_tmap(&tm_wd, w_down, E * d, I, 256);
+        if (!ok) return EXFOLD_ERR_CUDA;
+    }
+
+    EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
+
+    PrefillRouteParams rp{};
+    rp.logits = logits; rp.S = tables->S; rp.L = tables->L; rp.lnh = tables->lnh;
+    rp.T = T; rp.N = N; rp.K = K; rp.Kp = Kp;
+    rp.ids = at<int32_t>(ws, pl.ids); rp.w = at<float>(ws, pl.w);
+    rp.omit_src = at<int32_t>(ws, pl.omit_src); rp.omit_tgt = at<int32_t>(ws, pl.omit_tgt);
+    rp.block_hist = at<int32_t>(ws, pl.block_hist);
+    EXFOLD_CUDA(launch_prefill_route(rp, s));
+
+    const int nblk = (int)((T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
+    PrefillSortParams sp{};
+    sp.T = T; sp.N = N; sp.n_shared = l.n_shared; sp.Kp = Kp; sp.nblk = nblk;
+    sp.block_hist = rp.block_hist; sp.offsets = at<int32_t>(ws, pl.offsets);
+    sp.work_start = at<int32_t>(ws, pl.work_start); sp.totals = at<int32_t>(ws, pl.totals);
+    EXFOLD_CUDA(launch_prefill_sort(sp, s));
+
+    PrefillScatterParams cp{};
+    cp.T = T; cp.N = N; cp.n_shared = l.n_shared; cp.Kp = Kp; cp.d_bytes = bf16 ? d * 2 : 0;
+    cp.ids = rp.ids; cp.w = rp.w; cp.block_hist = rp.block_hist; cp.offsets = sp.offsets;
+    cp.x = x; cp.xs = bf16 ? at<char>(ws, pl.xs) : nullptr;
+    cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
+    cp.row_w = at<float>(ws, pl.row_w); cp.row_exp = at<int32_t>(ws, pl.row_exp);
+    EXFOLD_CUDA(launch_prefill_scatter(cp, s));
+
+    if (bf16) {
+        if (!direct) EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.y32), 0, (size_t)T * d * 4, s));
+        GroupedGemmParams g{};
+        g.tm_a = tm_xs; g.tm_a2 = tm_x; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu;
+        g.offsets = sp.offsets; g.work_start = sp.work_start; g.G = G; g.n_routed = N; g.R = (int)R;
+        g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128;
+        g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = cp.row_tok; g.row_w = cp.row_w;
+        g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
+        const int64_t max_tiles = Rtot / kTileM + G;
+        int grid1 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
+        EXFOLD_CUDA(launch_grouped_gemm1(g, grid1, s));
+        g.tm_a = tm_h; g.tm_b0 = tm_wd; g.n_ntiles = (d + 255) / 256;
+        g.y32 = direct ? nullptr : at<float>(ws, pl.y32);
+        g.y = reinterpret_cast<__nv_bfloat16*>(y);
+        int grid2 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
+        EXFOLD_CUDA(launch_grouped_gemm2(g, grid2, s));
+        if (!direct) EXFOLD_CUDA(launch_convert_bf16(at<float>(ws, pl.y32), T * d, y, s));
+    } else {
+        SimtFfnParams fp{};
+        fp.x = x; fp.wg = w_gate; fp.wu = w_up; fp.wd = w_down; fp.dtype = l.dtype; fp.d = d; fp.I = I;
+        fp.T = T; fp.Kr = Kp; fp.n_shared = l.n_shared; fp.N = N; fp.ids = rp.ids; fp.out = at<float>(ws, pl.out);
+        EXFOLD_CUDA(launch_simt_ffn(fp, s));
+        EXFOLD_CUDA(launch_combine_routes(fp.out, rp.w, T, Kp, d, l.n_shared, y, l.dtype, s));
+    }
+    if (meta) {
+        if ((rc = copy_meta(meta->ids, rp.ids, (size_t)R * 4, s))) return rc;
+        if ((rc = copy_meta(meta->w, rp.w, (size_t)R * 4, s))) return rc;
+        if ((rc = copy_meta(meta->omit_src, rp.omit_src, (size_t)T * (K - Kp) * 4, s))) return rc;
+        if ((rc = copy_meta(meta->omit_tgt, rp.omit_tgt, (size_t)T * (K - Kp) * 4, s))) return rc;
+        if ((rc = copy_meta(meta->perm, cp.perm, (size_t)R * 4, s))) return rc;
+        if ((rc = copy_meta(meta->offsets, sp.offsets, (size_t)(N + 1) * 4, s))) return rc;
+    }
+    return EXFOLD_OK;
+}
+
+int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* logits, int64_t B, const void* w_gate,
+                      const void* w_up, const void* w_down, const exfold_tables* tables, int32_t pool_m, void* y,
+                      const exfold_decode_meta* meta, void* ws, size_t ws_bytes, void* cuda_stream) {
+    int rc = check_common(layer, x, logits, B, w_gate, w_up, w_down, tables, y, ws);
+    if (rc != EXFOLD_OK) return rc;
+    const exfold_layer& l = *layer;
+    if (pool_m < 1 || pool_m > l.n_experts) return EXFOLD_ERR_INVALID_ARG;
+    if (B > kMaxDecodeBatch || B * l.top_k > 4096) return EXFOLD_ERR_UNSUPPORTED;
+    const int N = l.n_experts, K = l.top_k, d = l.hidden, I = l.inter, G = N + l.n_shared;
+    const Plan pl = make_plan(l, B, K);
+    if (ws_bytes < pl.total) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const bool bf16 = l.dtype == EXFOLD_BF16;
+    const int max_rows = (int)(B * K + B * l.n_shared);
+    int NB = (int)((B + 15) / 16 * 16);
+    if (NB < 16) NB = 16;
+
+    CUtensorMap tm_xs, tm_wg, tm_wu, tm_h, tm_wd;
+    if (bf16) {
+        const uint64_t E = (uint64_t)G;
+        bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)max_rows, d, NB) &&
+                  make_tmap(&tm_wg, w_gate, E * I, d, 128) && make_tmap(&tm_wu, w_up, E * I, d, 128) &&
+                  make_tmap(&tm_h, at<char>(ws, pl.H), (uint64_t)max_rows, I, NB) &&
+                  make_tmap(&tm_wd, w_down, E * d, I, 128);
+        if (!ok) return EXFOLD_ERR_CUDA;
+    }
+    EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
+
+    DecodeRouteParams rp{};
+    rp.logits = logits; rp.S = tables->S; rp.L = tables->L; rp.h = tables->h;
+    rp.B = (int)B; rp.N = N; rp.K = K; rp.M = pool_m; rp.n_shared = l.n_shared;
+    rp.pool_ids = at<int32_t>(ws, pl.pool_ids); rp.pool_size = at<int32_t>(ws, pl.pool_size);
+    rp.pool_mask = at<uint32_t>(ws, pl.pool_mask); rp.ids = at<int32_t>(ws, pl.ids); rp.w = at<float>(ws, pl.w);
+    rp.target = at<int32_t>(ws, pl.target); rp.scale = at<float>(ws, pl.scale);
+    rp.row_tok = at<int32_t>(ws, pl.row_tok); rp.row_w = at<float>(ws, pl.row_w);
+    rp.grp_expert = at<int32_t>(ws, pl.grp_expert); rp.grp_off = at<int32_t>(ws, pl.grp_off);
+    rp.n_groups = at<int32_t>(ws, pl.n_groups);
+    EXFOLD_CUDA(launch_decode_route(rp, s));
+
+    if (bf16) {
+        EXFOLD_CUDA(launch_gather_rows(x, rp.row_tok, rp.n_groups + 1, max_rows, d * 2, at<char>(ws, pl.xs),
+                                       at<float>(ws, pl.y32), (int)B, d, s));
+        DecodeFfnParams f{};
+        f.tm_w0 = tm_wg; f.tm_w1 = tm_wu; f.tm_act = tm_xs;
+        f.grp_expert = rp.grp_expert; f.grp_off = rp.grp_off; f.n_groups = rp.n_groups;
+        f.row_tok = rp.row_tok; f.row_w = rp.row_w; f.d = d; f.I = I; f.NB = NB; f.ksplit = 1;
+        f.max_groups = std::min(pool_m, N) + l.n_shared;
+        f.H = at<__nv_bfloat16>(ws, pl.H); f.y32 = at<float>(ws, pl.y32); f.status = at<DeviceStatus>(ws, pl.status);
+        const int sms = sm_count();
+        int items1 = f.max_groups * ((I + 127) / 128);
+        EXFOLD_CUDA(launch_decode_gateup(f, std::min(sms, items1), s));
+        f.tm_w0 = tm_wd; f.tm_act = tm_h;
+        const int n_ds = (d + 127) / 128, nkb = I / 64;
+        int ks = (2 * sms + f.max_groups * n_ds - 1) / (f.max_groups * n_ds);
+        if (ks > nkb / 4) ks = nkb / 4;
+        if (ks < 1) ks = 1;
+        f.ksplit = ks;
+        int items2 = f.max_groups * n_ds * ks;
+        EXFOLD_CUDA(launch_decode_down(f, std::min(sms, items2), s));
+        EXFOLD_CUDA(launch_convert_bf16(at<float>(ws, pl.y32), B * d, y, s));
+    } else {
+        SimtFfnParams fp{};
+        fp.x = x; fp.wg = w_gate; fp.wu = w_up; fp.wd = w_down; fp.dtype = l.dtype; fp.d = d; fp.I = I;
+        fp.T = B; fp.Kr = K; fp.n_shared = l.n_shared; fp.N = N; fp.ids = rp.ids; fp.out = at<float>(ws, pl.out);
+        EXFOLD_CUDA(launch_simt_ffn(fp, s));
+        EXFOLD_CUDA(launch_combine_routes(fp.out, rp.w, B, K, d, l.n_shared, y, l.dtype, s));
+    }
+    if (meta) {
+        if ((rc = copy_meta(meta->pool_ids, rp.pool_ids, (size_t)pool_m * 4, s))) return rc;
+        if ((rc = copy_meta(meta->pool_size, rp.pool_size, 4, s))) return rc;
+        if ((rc = copy_meta(meta->pool_mask, rp.pool_mask, (size_t)((N + 31) / 32) * 4, s))) return rc;
+        if ((rc = copy_meta(meta->ids, rp.ids, (size_t)B * K * 4, s))) return rc;
+        if ((rc = copy_meta(meta->w, rp.w, (size_t)B * K * 4, s))) return rc;
+        if ((rc = copy_meta(meta->target, rp.target, (size_t)N * 4, s))) return rc;
+        if ((rc = copy_meta(meta->scale, rp.scale, (size_t)N * 4, s))) return rc;
+    }
+    return EXFOLD_OK;
+}
+
+int exfold_calibrate(const exfold_layer* layer, const void* x_cal, const float* logits_cal, int64_t m,
+                     const void* w_gate, const void* w_up, const void* w_down, const exfold_calib_opts* opts,
+                     exfold_tables* out, void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (!valid_layer(layer) || !x_cal || !w_gate || !w_up || !w_down || !opts || !out || !ws)
+        return EXFOLD_ERR_INVALID_ARG;
+    if (!out->S || !out->L || !out->h || !out->lnh) return EXFOLD_ERR_INVALID_ARG;
+    if (m < 1 || m > (int64_t)1 << 22) return EXFOLD_ERR_INVALID_ARG;
+    if (opts->mode != 0 && opts->mode != 1) return EXFOLD_ERR_INVALID_ARG;
+    if (opts->mode == 0 && !logits_cal) return EXFOLD_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ws) & 255) != 0) return EXFOLD_ERR_INVALID_ARG;
+    const exfold_layer& l = *layer;
+    const int N = l.n_experts, K = l.top_k, d = l.hidden, I = l.inter;
+    const int Ke = opts->mode == 1 ? N : K;
+    exfold_layer lc = l;
+    lc.n_shared = 0;  // the shared expert is never folded, so it is not calibrated
+    const Plan pl = make_plan(lc, m, Ke);
+    if (ws_bytes < pl.total) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+
+    EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
+    int32_t* ids = at<int32_t>(ws, pl.ids);
+    if (opts->mode == 0) {
+        // Top-K in router order: the prefill route kernel with K' = K and a zero ln(h) table
+        EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.zeros), 0, (size_t)N * 4, s));
+        PrefillRouteParams rp{};
+        rp.logits = logits_cal; rp.S = out->S; rp.L = out->L; rp.lnh = at<float>(ws, pl.zeros);
+        rp.T = m; rp.N = N; rp.K = K; rp.Kp = K; rp.ids = ids; rp.w = at<float>(ws, pl.w);
+        rp.omit_src = nullptr; rp.omit_tgt = nullptr; rp.block_hist = at<int32_t>(ws, pl.block_hist);
+        EXFOLD_CUDA(launch_prefill_route(rp, s));
+    } else {
+        EXFOLD_CUDA(launch_iota_ids(ids, m, N, s));
+    }
+    SimtFfnParams fp{};
+    fp.x = x_cal; fp.wg = w_gate; fp.wu = w_up; fp.wd = w_down; fp.dtype = l.dtype; fp.d = d; fp.I = I;
+    fp.T = m; fp.Kr = Ke; fp.n_shared = 0; fp.N = N; fp.ids = ids; fp.out = at<float>(ws, pl.out);
+    EXFOLD_CUDA(launch_simt_ffn(fp, s));
+
+    char* cb = at<char>(ws, pl.calib);
+    const size_t NN = (size_t)N * N;
+    EXFOLD_CUDA(cudaMemsetAsync(cb, 0, NN * (3 * 8 + 4) + (size_t)N * (8 + 4) + 256, s));
+    CalibStatsParams cs{};
+    cs.out = fp.out; cs.ids = ids; cs.m = m; cs.Ke = Ke; cs.d = d; cs.N = N;
+    cs.A = reinterpret_cast<double*>(cb); cs.Bv = cs.A + NN; cs.C = cs.Bv + NN;
+    cs.H = cs.C + NN;
+    cs.cnt = reinterpret_cast<int32_t*>(cs.H + N);
+    cs.hc = cs.cnt + NN;
+    int32_t* unobs = cs.hc + N;
+    EXFOLD_CUDA(launch_calib_stats(cs, s));
+    EXFOLD_CUDA(launch_calib_finalize(cs, *opts, out->S, out->L, out->h, out->lnh, out->n_obs, unobs, s));
+    int un = 0;
+    EXFOLD_CUDA(cudaMemcpyAsync(&un, unobs, 4, cudaMemcpyDeviceToHost, s));
+    EXFOLD_CUDA(cudaStreamSynchronize(s));
+    return un > 0 ? EXFOLD_WARN_UNOBSERVED_EXPERT : EXFOLD_OK;
+}
+
+int exfold_moe_prefill_host(const exfold_layer* layer, const void* x_host, const float* logits_host, int64_t T,
+                            const void* w_gate, const void* w_up, const void* w_down, const exfold_tables* tables,
+                            int32_t k_pre, void* y_host, const exfold_prefill_meta* meta, void* ws, size_t ws_bytes,
+                            void* cuda_stream) {
+    if (!valid_layer(layer) || !x_host || !logits_host || !y_host || !ws || T < 1) return EXFOLD_ERR_INVALID_ARG;
+    if (k_pre < 1 || k_pre > layer->top_k) return EXFOLD_ERR_INVALID_ARG;
+    const size_t main_bytes = exfold_workspace_bytes(layer, T, k_pre);
+    const size_t el = layer->dtype == EXFOLD_BF16 ? 2 : 4;
+    const size_t xb = (size_t)T * layer->hidden * el, lb = (size_t)T * layer->n_experts * 4;
+    if (ws_bytes < main_bytes + exfold_host_staging_bytes(layer, T)) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
+    char* stage = reinterpret_cast<char*>(ws) + main_bytes;
+    char* xd = stage;
+    char* yd = xd + align_up(xb, 256);
+    char* ld = yd + align_up(xb, 256);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    EXFOLD_CUDA(cudaMemcpyAsync(xd, x_host, xb, cudaMemcpyHostToDevice, s));
+    EXFOLD_CUDA(cudaMemcpyAsync(ld, logits_host, lb, cudaMemcpyHostToDevice, s));
+    int rc = exfold_moe_prefill(layer, xd, reinterpret_cast<const float*>(ld), T, w_gate, w_up, w_down, tables, k_pre,
+                                yd, meta, ws, main_bytes, cuda_stream);
+    if (rc != EXFOLD_OK) return rc;
+    EXFOLD_CUDA(cudaMemcpyAsync(y_host, yd, xb, cudaMemcpyDeviceToHost, s));
+    return EXFOLD_OK;
+}
+
+int exfold_moe_decode_host(const exfold_layer* layer, const void* x_host, const float* logits_host, int64_t B,
+                           const void* w_gate, const void* w_up, const void* w_down, const exfold_tables* tables,
+                           int32_t pool_m, void* y_host, const exfold_decode_meta* meta, void* ws, size_t ws_bytes,
+                           void* cuda_stream) {
+    if (!valid_layer(layer) || !x_host || !logits_host || !y_host || !ws || B < 1) return EXFOLD_ERR_INVALID_ARG;
+    const size_t main_bytes = exfold_workspace_bytes(layer, B, layer->top_k);
+    const size_t el = layer->dtype == EXFOLD_BF16 ? 2 : 4;
+    const size_t xb = (size_t)B * layer->hidden * el, lb = (size_t)B * layer->n_experts * 4;
+    if (ws_bytes < main_bytes + exfold_host_staging_bytes(layer, B)) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
+    char* stage = reinterpret_cast<char*>(ws) + main_bytes;
+    char* xd = stage;
+    char* yd = xd + align_up(xb, 256);
+    char* ld = yd + align_up(xb, 256);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    EXFOLD_CUDA(cudaMemcpyAsync(xd, x_host, xb, cudaMemcpyHostToDevice, s));
+    EXFOLD_CUDA(cudaMemcpyAsync(ld, logits_host, lb, cudaMemcpyHostToDevice, s));
+    int rc = exfold_moe_decode(layer, xd, reinterpret_cast<const float*>(ld), B, w_gate, w_up, w_down, tables, pool_m,
+                               yd, meta, ws, main_bytes, cuda_stream);
+    if (rc != EXFOLD_OK) return rc;
+    EXFOLD_CUDA(cudaMemcpyAsync(y_host, yd, xb, cudaMemcpyDeviceToHost, s));
+    return EXFOLD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,189 @@
+// Shared declarations of the folded-MoE CUDA library (sm_100a only).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/exfold.h"
+
+namespace exfold {
+
+// The first 256 bytes of every workspace hold the device status record.
+struct DeviceStatus {
+    int code;    // 0 or EXFOLD_ERR_DEVICE_TIMEOUT
+    int where;   // which wait gave up (kernel-specific tag)
+    int detail;  // block index
+    int pad[61];
+};
+static_assert(sizeof(DeviceStatus) == 256, "status record is 256 bytes");
+
+constexpr int kMaxExperts = 256;  // routed experts
+constexpr int kMaxTopK = 32;
+constexpr int kMaxGroups = kMaxExperts + 1;  // + shared expert
+constexpr int kTileM = 128;                  // token rows per prefill GEMM tile
+constexpr int kMaxDecodeBatch = 256;
+
+__device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
+    if (atomicCAS(&st->code, 0, EXFOLD_ERR_DEVICE_TIMEOUT) == 0) {
+        st->where = where;
+        st->detail = (int)blockIdx.x;
+    }
+}
+
+// host-side launch accounting
+void count_launch(int n = 1);
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---------------------------------------------------------------- routing (prefill)
+struct PrefillRouteParams {
+    const float* logits;  // [T][N]
+    const float* S;       // [N][N]
+    const float* L;       // [N][N]
+    const float* lnh;     // [N]
+    int64_t T;
+    int N, K, Kp;
+    int32_t* ids;       // [T][Kp]
+    float* w;           // [T][Kp]
+    int32_t* omit_src;  // [T][K-Kp] or null
+    int32_t* omit_tgt;  // [T][K-Kp] or null
+    int32_t* block_hist;  // [nblk][N]
+};
+constexpr int kRouteTokensPerBlock = 64;
+constexpr int kRouteThreads = 512;
+
+struct PrefillSortParams {
+    int64_t T;
+    int N, n_shared, Kp, nblk;
+    int32_t* block_hist;  // [nblk][N] in: counts, out: exclusive prefix over blocks
+    int32_t* offsets;     // [G+1] sorted-row offsets (G = N + n_shared)
+    int32_t* work_start;  // [G+1] prefix of row tiles per group
+    int32_t* totals;      // [4]: total row tiles, total rows
+};
+
+struct PrefillScatterParams {
+    int64_t T;
+    int N, n_shared, Kp, d_bytes;  // d_bytes: bytes of one x row (0: no gather)
+    const int32_t* ids;         // [T][Kp]
+    const float* w;             // [T][Kp]
+    const int32_t* block_hist;  // prefix form
+    const int32_t* offsets;
+    const void* x;      // [T][d]
+    void* xs;           // [R][d] gathered rows (may be null)
+    int32_t* perm;      // [R]
+    int32_t* row_tok;   // [R + T*n_shared]
+    float* row_w;       // [R + T*n_shared]
+    int32_t* row_exp;   // [R + T*n_shared]
+};
+
+cudaError_t launch_prefill_route(const PrefillRouteParams& p, cudaStream_t s);
+cudaError_t launch_prefill_sort(const PrefillSortParams& p, cudaStream_t s);
+cudaError_t launch_prefill_scatter(const PrefillScatterParams& p, cudaStream_t s);
+
+// ---------------------------------------------------------------- routing (decode)
+struct DecodeRouteParams {
+    const float* logits;  // [B][N]
+    const float* S;
+    const float* L;
+    const float* h;
+    int B, N, K, M, n_shared;
+    // metadata (workspace copies)
+    int32_t* pool_ids;    // [N] (-1 padded)
+    int32_t* pool_size;   // [1]
+    uint32_t* pool_mask;  // [8]
+    int32_t* ids;         // [B][K]
+    float* w;             // [B][K]
+    int32_t* target;      // [N]
+    float* scale;         // [N]
+    // execution lists: rows sorted by pool rank (then shared expert), duplicates merged
+    int32_t* row_tok;     // [B*K + B]
+    float* row_w;         // [B*K + B]
+    int32_t* grp_expert;  // [N+1] expert id of each group (pool order; shared last)
+    int32_t* grp_off;     // [N+2] first row of each group
+    int32_t* n_groups;    // [2]: number of groups, total rows
+};
+cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s);
+cudaError_t launch_gather_rows(const void* x, const int32_t* row_tok, const int32_t* n_rows_ptr, int max_rows,
+                               int row_bytes, void* xs, float* y32, int zero_rows, int zero_row_floats,
+                               cudaStream_t s);
+
+// ---------------------------------------------------------------- SIMT expert FFN (fp32 accumulate)
+struct SimtFfnParams {
+    const void* x;  // [T][d]
+    const void* wg;
+    const void* wu;
+    const void* wd;
+    int dtype, d, I;
+    int64_t T;           // tokens
+    int Kr;              // routes per token; row r < T*Kr is route (r / Kr, r % Kr)
+    int n_shared, N;     // rows T*Kr + i run the shared expert (index N) on token i
+    const int32_t* ids;  // [T][Kr] expert of each route
+    float* out;          // [T*Kr + T*n_shared][d] unweighted expert outputs
+};
+cudaError_t launch_simt_ffn(const SimtFfnParams& p, cudaStream_t s);
+// y[i] = sum_j w[i][j] out[i*Kr+j] (+ out[T*Kr+i] for the shared expert); y in the layer dtype
+cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, int Kr, int d, int n_shared,
+                                  void* y, int dtype, cudaStream_t s);
+cudaError_t launch_convert_bf16(const float* y32, int64_t n, void* y, cudaStream_t s);
+
+// ---------------------------------------------------------------- calibration
+struct CalibStatsParams {
+    const float* out;    // [m][Ke][d] expert outputs
+    const int32_t* ids;  // [m][Ke]
+    int64_t m;
+    int Ke, d, N;
+    double* A;  // [N][N]
+    double* Bv;
+    double* C;
+    int32_t* cnt;  // [N][N]
+    double* H;     // [N]
+    int32_t* hc;   // [N]
+};
+cudaError_t launch_calib_stats(const CalibStatsParams& p, cudaStream_t s);
+cudaError_t launch_calib_finalize(const CalibStatsParams& p, const exfold_calib_opts& o, float* S, float* L,
+                                  float* h, float* lnh, int32_t* n_obs, int32_t* unobserved, cudaStream_t s);
+cudaError_t launch_iota_ids(int32_t* ids, int64_t m, int N, cudaStream_t s);
+
+// ---------------------------------------------------------------- tcgen05 grouped GEMMs (bf16)
+struct GroupedGemmParams {
+    CUtensorMap tm_a;    // GEMM-1: gathered rows Xs [R][d]; GEMM-2: H [Rtot][I]
+    CUtensorMap tm_a2;   // GEMM-1: x [T][d] for the shared expert's rows
+    CUtensorMap tm_b0;   // GEMM-1: W_gate as [(E*I)][d]; GEMM-2: W_down as [(E*d)][I]
+    CUtensorMap tm_b1;   // GEMM-1: W_up
+    const int32_t* offsets;     // [G+1]
+    const int32_t* work_start;  // [G+1] prefix of row tiles
+    int G;                      // groups (N + n_shared)
+    int n_routed;               // N
+    int R;                      // routed rows (shared rows start here)
+    int d, I;
+    int n_ntiles;               // column tiles
+    // epilogues
+    __nv_bfloat16* H;           // GEMM-1 out [Rtot][I]
+    const int32_t* row_tok;     // GEMM-2
+    const float* row_w;         // GEMM-2
+    float* y32;                 // GEMM-2 accumulate target (null: direct bf16 store)
+    __nv_bfloat16* y;           // GEMM-2 direct target
+    DeviceStatus* status;
+};
+cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s);
+cudaError_t launch_grouped_gemm2(const GroupedGemmParams& p, int grid, cudaStream_t s);
+
+struct DecodeFfnParams {
+    CUtensorMap tm_w0;  // gate/up kernel: W_gate [(E*I)][d]; down kernel: W_down [(E*d)][I]
+    CUtensorMap tm_w1;  // gate/up kernel: W_up
+    CUtensorMap tm_act; // gate/up kernel: Xs [rows][d]; down kernel: H [rows][I]; box rows = NB
+    const int32_t* grp_expert;
+    const int32_t* grp_off;
+    const int32_t* n_groups;
+    const int32_t* row_tok;
+    const float* row_w;
+    int d, I, NB, ksplit, max_groups;
+    __nv_bfloat16* H;  // [rows][I]
+    float* y32;        // [B][d]
+    DeviceStatus* status;
+};
+cudaError_t launch_decode_gateup(const DecodeFfnParams& p, int grid, cudaStream_t s);
+cudaError_t launch_decode_down(const DecodeFfnParams& p, int grid, cudaStream_t s);
+
+}  // namespace exfold

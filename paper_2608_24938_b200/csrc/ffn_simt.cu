@@ -1,0 +1,142 @@
+// SIMT (CUDA-core) expert FFN with fp32 accumulation, one CTA per route (Eq. 1).
+// Serves the fp32 layers end to end (tensor cores would round fp32 inputs), the
+// calibration pass (which needs each routed expert's unweighted output) and small
+// on-device cross-checks of the bf16 tensor-core path. Also the final combine /
+// conversion kernels (Eq. 3 / Eq. 4 weighted sums).
+#include "common.cuh"
+
+namespace exfold {
+
+namespace {
+
+__device__ __forceinline__ float ldf(const float* p, size_t i) { return __ldg(p + i); }
+__device__ __forceinline__ float ldf(const __nv_bfloat16* p, size_t i) {
+    return __bfloat162float(p[i]);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) simt_ffn_kernel(SimtFfnParams p) {
+    extern __shared__ float sm[];
+    float* xs = sm;          // [d]
+    float* act = sm + p.d;   // [I]
+    const int64_t row = blockIdx.x;
+    const int64_t n_routed = p.T * p.Kr;
+    int64_t tok;
+    int e;
+    if (row < n_routed) {
+        tok = row / p.Kr;
+        e = p.ids[row];
+    } else {
+        tok = row - n_routed;
+        e = p.N;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const T* x = reinterpret_cast<const T*>(p.x) + (size_t)tok * p.d;
+    for (int c = threadIdx.x; c < p.d; c += blockDim.x) xs[c] = ldf(x, c);
+    __syncthreads();
+    const T* wg = reinterpret_cast<const T*>(p.wg) + (size_t)e * p.I * p.d;
+    const T* wu = reinterpret_cast<const T*>(p.wu) + (size_t)e * p.I * p.d;
+    const T* wd = reinterpret_cast<const T*>(p.wd) + (size_t)e * p.d * p.I;
+    for (int j = warp; j < p.I; j += nwarps) {
+        float g = 0.f, u = 0.f;
+        const size_t base = (size_t)j * p.d;
+        for (int c = lane; c < p.d; c += 32) {
+            float xv = xs[c];
+            g = fmaf(ldf(wg, base + c), xv, g);
+            u = fmaf(ldf(wu, base + c), xv, u);
+        }
+        g = warp_sum(g);
+        u = warp_sum(u);
+        if (lane == 0) act[j] = (g / (1.0f + expf(-g))) * u;
+    }
+    __syncthreads();
+    float* out = p.out + (size_t)row * p.d;
+    for (int r = warp; r < p.d; r += nwarps) {
+        float o = 0.f;
+        const size_t base = (size_t)r * p.I;
+        for (int j = lane; j < p.I; j += 32) o = fmaf(ldf(wd, base + j), act[j], o);
+        o = warp_sum(o);
+        if (lane == 0) out[r] = o;
+    }
+}
+
+// y[i][c] = sum_j w[i][j] out[i*Kr+j][c] (+ out[T*Kr + i][c] for the shared expert), slot order
+template <typename T>
+__global__ void combine_routes_kernel(const float* __restrict__ out, const float* __restrict__ w, int64_t Tn,
+                                      int Kr, int d, int n_shared, T* __restrict__ y) {
+    const int64_t i = blockIdx.x;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        float acc = 0.f;
+        for (int j = 0; j < Kr; ++j) acc = fmaf(w[i * Kr + j], out[(size_t)(i * Kr + j) * d + c], acc);
+        if (n_shared) acc += out[(size_t)(Tn * Kr + i) * d + c];
+        if constexpr (sizeof(T) == 2) y[(size_t)i * d + c] = __float2bfloat16_rn(acc);
+        else y[(size_t)i * d + c] = acc;
+    }
+}
+
+__global__ void convert_bf16_kernel(const float4* __restrict__ src, int64_t n4, uint2* __restrict__ dst) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (; i < n4; i += stride) {
+        float4 v = src[i];
+        __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y);
+        __nv_bfloat162 b = __floats2bfloat162_rn(v.z, v.w);
+        uint2 o;
+        o.x = *reinterpret_cast<uint32_t*>(&a);
+        o.y = *reinterpret_cast<uint32_t*>(&b);
+        dst[i] = o;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_simt_ffn(const SimtFfnParams& p, cudaStream_t s) {
+    const int64_t rows = p.T * p.Kr + p.T * p.n_shared;
+    if (rows == 0) return cudaSuccess;
+    const size_t smem = (size_t)(p.d + p.I) * sizeof(float);
+    cudaError_t err;
+    if (p.dtype == EXFOLD_BF16) {
+        err = cudaFuncSetAttribute(simt_ffn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)smem);
+        if (err != cudaSuccess) return err;
+        simt_ffn_kernel<__nv_bfloat16><<<(unsigned)rows, 256, smem, s>>>(p);
+    } else {
+        err = cudaFuncSetAttribute(simt_ffn_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        simt_ffn_kernel<float><<<(unsigned)rows, 256, smem, s>>>(p);
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, int Kr, int d, int n_shared,
+                                  void* y, int dtype, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    if (dtype == EXFOLD_BF16)
+        combine_routes_kernel<__nv_bfloat16><<<(unsigned)T, 256, 0, s>>>(out, w, T, Kr, d, n_shared,
+                                                                         reinterpret_cast<__nv_bfloat16*>(y));
+    else
+        combine_routes_kernel<float><<<(unsigned)T, 256, 0, s>>>(out, w, T, Kr, d, n_shared,
+                                                                 reinterpret_cast<float*>(y));
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_convert_bf16(const float* y32, int64_t n, void* y, cudaStream_t s) {
+    if (n == 0) return cudaSuccess;
+    const int64_t n4 = n / 4;  // n is a multiple of 64 (d is)
+    int blocks = (int)((n4 + 255) / 256);
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    convert_bf16_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(y32), n4,
+                                               reinterpret_cast<uint2*>(y));
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace exfold

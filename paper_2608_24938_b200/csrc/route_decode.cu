@@ -1,0 +1,296 @@
+// Decode routing: batch-level expert pool (Eq. 11), minimum-loss targets (Eq. 12) and the
+// in-place remap of every routed slot (Eq. 14), in ONE CTA: B*K <= 4096 slots live in
+// shared memory. Also builds the execution lists for the weight-streaming FFN: rows sorted
+// by pool rank, duplicate (token, expert) slots merged ("routes folded into the same target
+// are coalesced before expert computation").
+#include "common.cuh"
+
+namespace exfold {
+
+namespace {
+
+constexpr int kDecThreads = 1024;
+constexpr int kDecMaxSlots = 4096;
+
+struct DecSmem {
+    double w64[kDecMaxSlots];
+    int ids[kDecMaxSlots];
+    float wrm[kDecMaxSlots];  // remapped weights
+    double score[kMaxExperts];
+    int in_union[kMaxExperts];
+    int rank_of[kMaxExperts];   // pool rank or -1
+    int pool[kMaxExperts];      // pool ids by rank
+    int target[kMaxExperts];
+    float scale[kMaxExperts];
+    int gcnt[kMaxExperts + 2];
+    int goff[kMaxExperts + 2];
+    int P;
+};
+
+template <int NPL>
+__global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRouteParams p) {
+    extern __shared__ __align__(16) unsigned char smraw[];
+    DecSmem& sm = *reinterpret_cast<DecSmem*>(smraw);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int kWarps = kDecThreads / 32;
+    const int B = p.B, N = p.N, K = p.K, M = p.M;
+
+    // ---- Eq. 2 per token (warp per token), weights in double
+    for (int i = warp; i < B; i += kWarps) {
+        const float* r = p.logits + (size_t)i * N;
+        float v[NPL];
+        uint32_t used = 0;
+#pragma unroll
+        for (int q = 0; q < NPL; ++q) {
+            int e = lane + 32 * q;
+            v[q] = e < N ? r[e] : -INFINITY;
+            if (e >= N) used |= 1u << q;
+        }
+        int my_id = -1;
+        float my_r = 0.f;
+        for (int k = 0; k < K; ++k) {
+            float bv = -INFINITY;
+            int be = 0x7fffffff;
+#pragma unroll
+            for (int q = 0; q < NPL; ++q) {
+                bool free_q = !((used >> q) & 1u);
+                if (free_q && (be == 0x7fffffff || v[q] > bv)) {
+                    bv = v[q];
+                    be = lane + 32 * q;
+                }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                int oe = __shfl_xor_sync(0xffffffffu, be, off);
+                if (oe != 0x7fffffff && (be == 0x7fffffff || ov > bv || (ov == bv && oe < be))) {
+                    bv = ov;
+                    be = oe;
+                }
+            }
+            if ((be & 31) == lane) used |= 1u << (be >> 5);
+            if (lane == k) {
+                my_id = be;
+                my_r = bv;
+            }
+        }
+        const float rmax = __shfl_sync(0xffffffffu, my_r, 0);
+        double ex = lane < K ? exp((double)my_r - (double)rmax) : 0.0;
+        double sum = 0.0;
+        for (int k = 0; k < K; ++k) sum += __shfl_sync(0xffffffffu, ex, k);  // slot order, like the definition
+        if (lane < K) {
+            sm.ids[i * K + lane] = my_id;
+            sm.w64[i * K + lane] = ex / sum;
+        }
+    }
+    __syncthreads();
+
+    // ---- Eq. 11: union and score_e = h_e * sum_i w_{i,e} (double; fixed reduction order)
+    const int nslots = B * K;
+    for (int e = warp; e < N; e += kWarps) {
+        double acc = 0.0;
+        int cnt = 0;
+        for (int s = lane; s < nslots; s += 32)
+            if (sm.ids[s] == e) {
+                acc += sm.w64[s];
+                cnt++;
+            }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+        }
+        if (lane == 0) {
+            sm.score[e] = acc * (double)p.h[e];
+            sm.in_union[e] = cnt > 0;
+        }
+    }
+    __syncthreads();
+    // pool = best min(M, |U|) experts of the union by (score desc, id asc)
+    {
+        int e = threadIdx.x;
+        int in_u = (e < N) ? sm.in_union[e] : 0;
+        int usize = __syncthreads_count(in_u);
+        if (e < N) {
+            int rk = -1;
+            if (in_u) {
+                rk = 0;
+                const double se = sm.score[e];
+                for (int o = 0; o < N; ++o)
+                    if (sm.in_union[o] && (sm.score[o] > se || (sm.score[o] == se && o < e))) rk++;
+                if (rk >= M) rk = -1;
+            }
+            sm.rank_of[e] = rk;
+            if (rk >= 0) sm.pool[rk] = e;
+        }
+        if (threadIdx.x == 0) sm.P = usize < M ? usize : M;
+    }
+    __syncthreads();
+    const int P = sm.P;
+    // ---- Eq. 12 for every source expert: itself if in the pool, else its min-loss pool expert
+    for (int s = warp; s < N; s += kWarps) {
+        if (sm.rank_of[s] >= 0) {
+            if (lane == 0) {
+                sm.target[s] = s;
+                sm.scale[s] = 1.0f;
+            }
+            continue;
+        }
+        float bl = INFINITY;
+        int bt = 0x7fffffff;
+        for (int j = lane; j < P; j += 32) {
+            int t = sm.pool[j];
+            float l = __ldg(p.L + (size_t)s * N + t);
+            if (bt == 0x7fffffff || l < bl || (l == bl && t < bt)) {
+                bl = l;
+                bt = t;
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            float ol = __shfl_xor_sync(0xffffffffu, bl, off);
+            int ot = __shfl_xor_sync(0xffffffffu, bt, off);
+            if (ot != 0x7fffffff && (bt == 0x7fffffff || ol < bl || (ol == bl && ot < bt))) {
+                bl = ol;
+                bt = ot;
+            }
+        }
+        if (lane == 0) {
+            sm.target[s] = bt;
+            sm.scale[s] = __ldg(p.S + (size_t)s * N + bt);
+        }
+    }
+    __syncthreads();
+    // ---- Eq. 14: remap every slot in place; [B][K] layout kept
+    for (int s = threadIdx.x; s < nslots; s += kDecThreads) {
+        int e = sm.ids[s];
+        int t = sm.target[e];
+        float wv = (float)(sm.w64[s] * (double)sm.scale[e]);
+        sm.ids[s] = t;
+        sm.wrm[s] = wv;
+        p.ids[s] = t;
+        p.w[s] = wv;
+    }
+    for (int e = threadIdx.x; e < N; e += kDecThreads) {
+        p.target[e] = sm.target[e];
+        p.scale[e] = sm.scale[e];
+        p.pool_ids[e] = e < P ? sm.pool[e] : -1;
+    }
+    if (threadIdx.x < 8) {
+        uint32_t m = 0;
+        for (int b = 0; b < 32; ++b) {
+            int e = threadIdx.x * 32 + b;
+            if (e < N && sm.rank_of[e] >= 0) m |= 1u << b;
+        }
+        p.pool_mask[threadIdx.x] = m;
+    }
+    if (threadIdx.x == 0) *p.pool_size = P;
+    __syncthreads();
+    // ---- execution lists: one row per distinct (token, pool expert), grouped by pool rank
+    for (int pass = 0; pass < 2; ++pass) {
+        for (int g = warp; g < P; g += kWarps) {
+            const int t = sm.pool[g];
+            int run = pass ? sm.goff[g] : 0;
+            for (int i0 = 0; i0 < B; i0 += 32) {
+                int i = i0 + lane;
+                bool has = false;
+                float ws = 0.f;
+                if (i < B)
+                    for (int k = 0; k < K; ++k)
+                        if (sm.ids[i * K + k] == t) {
+                            ws = has ? __fadd_rn(ws, sm.wrm[i * K + k]) : sm.wrm[i * K + k];
+                            has = true;
+                        }
+                unsigned m = __ballot_sync(0xffffffffu, has);
+                if (pass && has) {
+                    int q = run + __popc(m & ((1u << lane) - 1u));
+                    p.row_tok[q] = i;
+                    p.row_w[q] = ws;
+                }
+                run += __popc(m);
+            }
+            if (!pass && lane == 0) sm.gcnt[g] = run;
+        }
+        __syncthreads();
+        if (!pass) {
+            if (threadIdx.x == 0) {
+                int off = 0;
+                for (int g = 0; g < P; ++g) {
+                    sm.goff[g] = off;
+                    off += sm.gcnt[g];
+                }
+                sm.goff[P] = off;
+                if (p.n_shared) sm.goff[P + 1] = off + B;
+            }
+            __syncthreads();
+        }
+    }
+    const int G = P + (p.n_shared ? 1 : 0);
+    for (int g = threadIdx.x; g <= G; g += kDecThreads) {
+        p.grp_off[g] = sm.goff[g];
+        if (g < G) p.grp_expert[g] = g < P ? sm.pool[g] : N;
+    }
+    if (p.n_shared)
+        for (int i = threadIdx.x; i < B; i += kDecThreads) {
+            p.row_tok[sm.goff[P] + i] = i;
+            p.row_w[sm.goff[P] + i] = 1.0f;
+        }
+    if (threadIdx.x == 0) {
+        p.n_groups[0] = G;
+        p.n_groups[1] = sm.goff[G];  // total rows
+    }
+}
+
+// xs[row] = x[row_tok[row]] for row < n_rows (device value); CTAs with blockIdx < zero_rows also
+// clear one row of the fp32 accumulator y32.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const void* __restrict__ x,
+                                                          const int32_t* __restrict__ row_tok,
+                                                          const int32_t* __restrict__ n_rows_ptr, int row_bytes,
+                                                          void* __restrict__ xs, float* __restrict__ y32,
+                                                          int zero_rows, int zero_row_floats) {
+    const int row = blockIdx.x;
+    if (y32 != nullptr && row < zero_rows) {
+        float4* z = reinterpret_cast<float4*>(y32 + (size_t)row * zero_row_floats);
+        for (int c = threadIdx.x; c < zero_row_floats / 4; c += blockDim.x) z[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (row >= *n_rows_ptr) return;
+    const uint4* src =
+        reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(x) + (size_t)row_tok[row] * row_bytes);
+    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<char*>(xs) + (size_t)row * row_bytes);
+    for (int c = threadIdx.x; c < (row_bytes >> 4); c += blockDim.x) dst[c] = __ldg(src + c);
+}
+
+}  // namespace
+
+cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s) {
+    const int npl = (p.N + 31) / 32;
+    const size_t smem = sizeof(DecSmem);
+    cudaError_t err = cudaSuccess;
+#define EXFOLD_DEC_LAUNCH(NPL)                                                                              \
+    err = cudaFuncSetAttribute(decode_route_kernel<NPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
+                               (int)smem);                                                                  \
+    if (err != cudaSuccess) return err;                                                                     \
+    decode_route_kernel<NPL><<<1, kDecThreads, smem, s>>>(p);
+    switch (npl) {
+        case 1: EXFOLD_DEC_LAUNCH(1) break;
+        case 2: EXFOLD_DEC_LAUNCH(2) break;
+        case 3: case 4: EXFOLD_DEC_LAUNCH(4) break;
+        default: EXFOLD_DEC_LAUNCH(8) break;
+    }
+#undef EXFOLD_DEC_LAUNCH
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather_rows(const void* x, const int32_t* row_tok, const int32_t* n_rows_ptr, int max_rows,
+                               int row_bytes, void* xs, float* y32, int zero_rows, int zero_row_floats,
+                               cudaStream_t s) {
+    int grid = max_rows > zero_rows ? max_rows : zero_rows;
+    if (grid == 0) return cudaSuccess;
+    gather_rows_kernel<<<grid, 256, 0, s>>>(x, row_tok, n_rows_ptr, row_bytes, xs, y32, zero_rows,
+                                            zero_row_floats);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace exfold

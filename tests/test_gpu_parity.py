@@ -1,0 +1,201 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs. Routing metadata bit-exact, outputs within the stated tolerances."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from harness import A, Case, check_decode_meta, check_output, check_prefill_meta
+
+pytestmark = pytest.mark.gpu
+
+TINY = si.CONFIGS["tiny"]
+
+
+def small_bf16(**kw):
+    base = dict(name="small", n_experts=16, n_shared=0, hidden=256, inter=384, top_k=4, dtype="bf16",
+                prefill_tokens=300, k_pre=(2,), decode_batch=24, pool_m=(6,), logits="zipf")
+    base.update(kw)
+    return si.LayerConfig(**base)
+
+
+def calibrated_tables(case, cfg, lam=1e-3):
+    xc = si.hidden_states(cfg, cfg.calib_tokens, "x_cal")
+    lc = si.router_logits(cfg, cfg.calib_tokens, "logits_cal")
+    cal = oracle.calibrate(A(xc), lc.numpy(), A(case.wg), A(case.wu), A(case.wd), cfg.n_experts, cfg.top_k, lam=lam)
+    return xc, lc, cal
+
+
+# ------------------------------------------------------------------ fp32 tiny layer (SIMT path)
+@pytest.mark.parametrize("correlated", [0.0, 0.8])
+def test_tiny_fp32_layer(correlated):
+    cfg = TINY
+    case = Case(cfg, std=0.02, correlated=correlated)
+    xc, lc, cal = calibrated_tables(case, cfg)
+    case.set_tables((cal["S"], cal["L"], cal["h"], cal["lnh"]))
+    if correlated:
+        off = ~np.eye(cfg.n_experts, dtype=bool)
+        assert np.abs(cal["S"][off]).mean() > 0.2   # folding matters in this variant
+    for Kp in (1, 2):
+        got, ref = case.run_prefill(Kp), case.oracle_prefill(Kp)
+        check_prefill_meta(got, ref)
+        check_output(got["y"], ref["y"], "f32")
+    for M in (4, 1, 8):
+        got, ref = case.run_decode(M), case.oracle_decode(M)
+        assert ref["min_gap"] > 1e-9, "degenerate input: pool boundary tie"
+        check_decode_meta(got, ref, M)
+        check_output(got["y"], ref["y"], "f32")
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_calibrate_matches_oracle(mode):
+    cfg = TINY
+    case = Case(cfg, std=0.02, correlated=0.8)
+    ex, dev = case.ex, case.dev
+    m, N, K = cfg.calib_tokens, cfg.n_experts, cfg.top_k
+    xc = si.hidden_states(cfg, m, "x_cal")
+    lc = si.router_logits(cfg, m, "logits_cal")
+    ref = oracle.calibrate(A(xc), lc.numpy(), A(case.wg), A(case.wu), A(case.wd), N, K, mode=mode)
+    S = torch.full((N, N), float("nan"), device=dev)
+    L, h, lnh = torch.full_like(S, float("nan")), torch.full((N,), float("nan"), device=dev), torch.empty(N, device=dev)
+    n_obs = torch.full((N, N), -1, dtype=torch.int32, device=dev)
+    ws = ex.alloc_workspace(case.layer, m, N if mode else K)
+    ws.fill_(0xFF)
+    rc = ex.exfold_calibrate(case.layer, xc.to(dev), lc.to(dev), case.d_wg, case.d_wu, case.d_wd,
+                             ex.make_tables(S, L, h, lnh, n_obs), ws, mode=mode)
+    assert rc == (1 if ref["unobserved"] else 0)
+    assert np.array_equal(n_obs.cpu().numpy(), ref["n_obs"])
+    np.testing.assert_allclose(S.cpu().numpy(), ref["S"], rtol=2e-5, atol=2e-6)
+    np.testing.assert_allclose(L.cpu().numpy(), ref["L"], rtol=1e-4, atol=2e-5)
+    np.testing.assert_allclose(h.cpu().numpy(), ref["h"], rtol=1e-5)
+    np.testing.assert_allclose(lnh.cpu().numpy(), ref["lnh"], rtol=1e-5, atol=1e-6)
+    assert (np.diag(S.cpu().numpy()) == 1).all() and (np.diag(L.cpu().numpy()) == 0).all()
+
+
+# ------------------------------------------------------------------ bf16 tensor-core path
+@pytest.mark.parametrize("Kp", [2, 1, 4])
+def test_bf16_prefill_small(Kp):
+    case = Case(small_bf16())
+    got, ref = case.run_prefill(Kp), case.oracle_prefill(Kp)
+    assert ref["mismatch"] == 0
+    check_prefill_meta(got, ref)
+    check_output(got["y"], ref["y"], "bf16")
+
+
+@pytest.mark.parametrize("M", [6, 1, 16])
+def test_bf16_decode_small(M):
+    case = Case(small_bf16())
+    got, ref = case.run_decode(M), case.oracle_decode(M)
+    assert ref["min_gap"] > 1e-9
+    check_decode_meta(got, ref, M)
+    check_output(got["y"], ref["y"], "bf16")
+
+
+def test_bf16_shared_expert_and_correlated_experts():
+    cfg = small_bf16(n_shared=1, n_experts=8, top_k=3, prefill_tokens=200, decode_batch=17)
+    case = Case(cfg, correlated=0.8)
+    got, ref = case.run_prefill(2), case.oracle_prefill(2)
+    check_prefill_meta(got, ref)
+    check_output(got["y"], ref["y"], "bf16")
+    got, ref = case.run_decode(3), case.oracle_decode(3)
+    check_decode_meta(got, ref, 3)
+    check_output(got["y"], ref["y"], "bf16")
+
+
+def test_bf16_several_tiles_and_ragged_tail():
+    """Groups of 0, 1, hundreds of rows; several 128-row tiles per expert; K and N tails."""
+    cfg = small_bf16(n_experts=8, hidden=512, inter=832, top_k=2, prefill_tokens=1111, decode_batch=64,
+                     logits="zipf", zipf_s=2.0)
+    case = Case(cfg)
+    lgm = case.lg.clone()
+    lgm[:, 5] = -50.0          # expert 5 receives no route at all
+    case.lg, case.d_lg = lgm, lgm.to(case.dev)
+    for Kp in (1, 2):
+        got, ref = case.run_prefill(Kp), case.oracle_prefill(Kp)
+        counts = np.diff(ref["offsets"])
+        assert counts[5] == 0 and counts.max() > 256
+        check_prefill_meta(got, ref)
+        check_output(got["y"], ref["y"], "bf16")
+    got, ref = case.run_decode(3), case.oracle_decode(3)
+    check_decode_meta(got, ref, 3)
+    check_output(got["y"], ref["y"], "bf16")
+
+
+@pytest.mark.parametrize("T", [1, 63, 129])
+def test_bf16_odd_token_counts(T):
+    cfg = small_bf16(prefill_tokens=T, decode_batch=min(T, 256))
+    case = Case(cfg)
+    got, ref = case.run_prefill(2), case.oracle_prefill(2)
+    check_prefill_meta(got, ref)
+    check_output(got["y"], ref["y"], "bf16")
+    got, ref = case.run_decode(4), case.oracle_decode(4)
+    check_decode_meta(got, ref, 4)
+    check_output(got["y"], ref["y"], "bf16")
+
+
+def test_full_budget_is_the_unfolded_layer():
+    """K' = K and M = N: no folding, output equals Eq. 3 computed by the oracle from Eq. 2's routes."""
+    cfg = small_bf16()
+    case = Case(cfg)
+    ids, w, _ = oracle.gate(case.lg.numpy(), cfg.top_k)
+    y_unf = oracle.moe_apply(A(case.x), A(case.wg), A(case.wu), A(case.wd), ids, w, cfg.n_experts)
+    got = case.run_prefill(cfg.top_k)
+    assert np.array_equal(np.sort(got["ids"], 1), np.sort(ids, 1))
+    check_output(got["y"], y_unf, "bf16")
+    idd, wd_, _ = oracle.gate(case.lgd.numpy(), cfg.top_k)
+    yd_unf = oracle.moe_apply(A(case.xd), A(case.wg), A(case.wu), A(case.wd), idd, wd_, cfg.n_experts)
+    gotd = case.run_decode(cfg.n_experts)
+    assert np.array_equal(gotd["ids"], idd)
+    np.testing.assert_allclose(gotd["w"], wd_, rtol=1e-6)
+    check_output(gotd["y"], yd_unf, "bf16")
+
+
+def test_decode_max_batch_and_all_unobserved_row():
+    cfg = small_bf16(n_experts=32, top_k=8, decode_batch=256, prefill_tokens=64)
+    case = Case(cfg)
+    S, L, h, lnh = [t.clone() for t in case.tables_host]
+    L[3, :] = 1e30
+    L[3, 3] = 0.0
+    S[3, :] = 0.0
+    S[3, 3] = 1.0
+    case.set_tables((S, L, h, lnh))
+    for M in (8, 20):
+        got, ref = case.run_decode(M), case.oracle_decode(M)
+        assert ref["min_gap"] > 1e-9
+        check_decode_meta(got, ref, M)
+        check_output(got["y"], ref["y"], "bf16")
+    got, ref = case.run_prefill(3), case.oracle_prefill(3)
+    check_prefill_meta(got, ref)
+    check_output(got["y"], ref["y"], "bf16")
+
+
+def test_results_are_reproducible_and_meta_is_optional():
+    case = Case(small_bf16())
+    a = case.run_prefill(2)
+    b = case.run_prefill(2)
+    for k in ("ids", "perm", "offsets", "omit_src", "omit_tgt"):
+        assert np.array_equal(a[k], b[k])
+    assert np.array_equal(a["w"], b["w"])
+    c = case.run_prefill(2, with_meta=False)
+    np.testing.assert_allclose(c["y"], a["y"], rtol=0, atol=2e-2 * np.abs(a["y"]).max())
+    d1, d2 = case.run_decode(6), case.run_decode(6, with_meta=False)
+    np.testing.assert_allclose(d2["y"], d1["y"], rtol=0, atol=2e-2 * np.abs(d1["y"]).max())
+
+
+def test_host_buffer_entry_points():
+    case = Case(small_bf16())
+    ex, cfg = case.ex, case.cfg
+    T, B, K = case.T, case.B, cfg.top_k
+    ws = ex.alloc_workspace(case.layer, max(T, B), K, host_staging=True)
+    xh, lh = case.x.pin_memory(), case.lg.pin_memory()
+    yh = torch.empty((T, cfg.hidden), dtype=torch.bfloat16).pin_memory()
+    ex.exfold_moe_prefill_host(case.layer, xh, lh, case.d_wg, case.d_wu, case.d_wd, case.tables, 2, yh, ws)
+    assert ex.exfold_device_status(ws) == 0
+    ref = case.oracle_prefill(2)
+    check_output(yh.float().numpy(), ref["y"], "bf16")
+    xdh, ldh = case.xd.pin_memory(), case.lgd.pin_memory()
+    ydh = torch.empty((B, cfg.hidden), dtype=torch.bfloat16).pin_memory()
+    ex.exfold_moe_decode_host(case.layer, xdh, ldh, case.d_wg, case.d_wu, case.d_wd, case.tables, 6, ydh, ws)
+    assert ex.exfold_device_status(ws) == 0
+    check_output(ydh.float().numpy(), case.oracle_decode(6)["y"], "bf16")
