@@ -181,6 +181,21 @@ const char *exfold_status_string(int status);
 /* Number of kernels of this library launched by this process so far (for launch accounting). */
 int64_t exfold_launch_count(void);
 
+/*
+ * Per-kernel timing for benchmarks (host-side state; not thread-safe; off by default).
+ * exfold_profile_enable(1) creates one CUDA event pair per kernel slot; while enabled, every
+ * launch of the serving calls is bracketed by event records on the call's stream.
+ * exfold_profile_read synchronises on the recorded events of the LAST call and writes, for
+ * each slot < n_slots, the elapsed milliseconds (or -1 if that kernel did not run in the last
+ * call). Slots: 0 prefill route/fold, 1 prefill scan, 2 prefill scatter+gather, 3 grouped GEMM-1
+ * (gate/up + SwiGLU), 4 grouped GEMM-2 (down + scatter-combine), 5 fp32->bf16 conversion,
+ * 6 decode pool/remap, 7 decode row gather, 8 decode gate/up stream, 9 decode down stream,
+ * 10 SIMT expert FFN, 11 SIMT combine. Returns EXFOLD_OK or EXFOLD_ERR_CUDA.
+ */
+#define EXFOLD_PROFILE_SLOTS 12
+int exfold_profile_enable(int enable);
+int exfold_profile_read(float *ms, int32_t n_slots);
+
 #ifdef __cplusplus
 }
 #endif

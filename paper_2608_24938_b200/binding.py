@@ -26,7 +26,10 @@ EXFOLD_WARN_UNOBSERVED_EXPERT = 1
 
 EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibrate", "exfold_moe_prefill",
            "exfold_moe_decode", "exfold_moe_prefill_host", "exfold_moe_decode_host", "exfold_device_status",
-           "exfold_status_string", "exfold_launch_count"]
+           "exfold_status_string", "exfold_launch_count", "exfold_profile_enable", "exfold_profile_read"]
+PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
+                 "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
+                 "simt_combine"]
 
 
 class exfold_layer(C.Structure):
@@ -80,6 +83,10 @@ def _load() -> C.CDLL:
     lib.exfold_status_string.argtypes = [C.c_int]
     lib.exfold_launch_count.restype = i64
     lib.exfold_launch_count.argtypes = []
+    lib.exfold_profile_enable.restype = C.c_int
+    lib.exfold_profile_enable.argtypes = [C.c_int]
+    lib.exfold_profile_read.restype = C.c_int
+    lib.exfold_profile_read.argtypes = [C.POINTER(C.c_float), i32]
     return lib
 
 
@@ -123,6 +130,20 @@ def exfold_status_string(code: int) -> str:
 
 def exfold_launch_count() -> int:
     return int(lib.exfold_launch_count())
+
+
+def exfold_profile_enable(enable: bool) -> int:
+    return int(lib.exfold_profile_enable(1 if enable else 0))
+
+
+def exfold_profile_read() -> dict:
+    """Milliseconds of each kernel of the last call (kernels that did not run are left out)."""
+    n = len(PROFILE_SLOTS)
+    buf = (C.c_float * n)()
+    rc = lib.exfold_profile_read(buf, n)
+    if rc != 0:
+        raise ExfoldError(rc, "exfold_profile_read")
+    return {PROFILE_SLOTS[i]: float(buf[i]) for i in range(n) if buf[i] >= 0}
 
 
 def exfold_workspace_bytes(layer: exfold_layer, max_tokens: int, routes_per_token: int) -> int:

@@ -13,6 +13,31 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 namespace {
 
+// ------------------------------------------------------------------ optional per-kernel event timing
+struct Profiler {
+    bool on = false;
+    cudaEvent_t beg[EXFOLD_PROFILE_SLOTS];
+    cudaEvent_t end[EXFOLD_PROFILE_SLOTS];
+    bool used[EXFOLD_PROFILE_SLOTS];
+} g_prof;
+
+struct ProfScope {  // records an event pair around one launch when profiling is enabled
+    int slot;
+    cudaStream_t s;
+    ProfScope(int slot_, cudaStream_t s_) : slot(slot_), s(s_) {
+        if (g_prof.on) cudaEventRecord(g_prof.beg[slot], s);
+    }
+    ~ProfScope() {
+        if (g_prof.on) {
+            cudaEventRecord(g_prof.end[slot], s);
+            g_prof.used[slot] = true;
+        }
+    }
+};
+void prof_reset() {
+    for (int i = 0; i < EXFOLD_PROFILE_SLOTS; ++i) g_prof.used[i] = false;
+}
+
 // ------------------------------------------------------------------ workspace plan
 struct Plan {
     size_t status, ids, w, omit_src, omit_tgt, block_hist, offsets, work_start, totals, perm, row_tok, row_w,
@@ -178,6 +203,35 @@ size_t exfold_host_staging_bytes(const exfold_layer* layer, int64_t max_tokens) 
 
 int64_t exfold_launch_count(void) { return g_launches.load(); }
 
+int exfold_profile_enable(int enable) {
+    if (enable && !g_prof.on) {
+        for (int i = 0; i < EXFOLD_PROFILE_SLOTS; ++i) {
+            if (cudaEventCreate(&g_prof.beg[i]) != cudaSuccess) return EXFOLD_ERR_CUDA;
+            if (cudaEventCreate(&g_prof.end[i]) != cudaSuccess) return EXFOLD_ERR_CUDA;
+        }
+        prof_reset();
+        g_prof.on = true;
+    } else if (!enable && g_prof.on) {
+        g_prof.on = false;
+        for (int i = 0; i < EXFOLD_PROFILE_SLOTS; ++i) {
+            cudaEventDestroy(g_prof.beg[i]);
+            cudaEventDestroy(g_prof.end[i]);
+        }
+    }
+    return EXFOLD_OK;
+}
+
+int exfold_profile_read(float* ms, int32_t n_slots) {
+    if (!ms || n_slots < 0) return EXFOLD_ERR_INVALID_ARG;
+    for (int i = 0; i < n_slots; ++i) {
+        ms[i] = -1.0f;
+        if (!g_prof.on || i >= EXFOLD_PROFILE_SLOTS || !g_prof.used[i]) continue;
+        if (cudaEventSynchronize(g_prof.end[i]) != cudaSuccess) return EXFOLD_ERR_CUDA;
+        if (cudaEventElapsedTime(&ms[i], g_prof.beg[i], g_prof.end[i]) != cudaSuccess) return EXFOLD_ERR_CUDA;
+    }
+    return EXFOLD_OK;
+}
+
 const char* exfold_status_string(int status) {
     switch (status) {
         case EXFOLD_OK: return "ok";
@@ -228,6 +282,7 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
         if (!ok) return EXFOLD_ERR_CUDA;
     }
 
+    prof_reset();
     EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
 
     PrefillRouteParams rp{};
@@ -236,14 +291,14 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     rp.ids = at<int32_t>(ws, pl.ids); rp.w = at<float>(ws, pl.w);
     rp.omit_src = at<int32_t>(ws, pl.omit_src); rp.omit_tgt = at<int32_t>(ws, pl.omit_tgt);
     rp.block_hist = at<int32_t>(ws, pl.block_hist);
-    EXFOLD_CUDA(launch_prefill_route(rp, s));
+    { ProfScope ps(0, s); EXFOLD_CUDA(launch_prefill_route(rp, s)); }
 
     const int nblk = (int)((T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
     PrefillSortParams sp{};
     sp.T = T; sp.N = N; sp.n_shared = l.n_shared; sp.Kp = Kp; sp.nblk = nblk;
     sp.block_hist = rp.block_hist; sp.offsets = at<int32_t>(ws, pl.offsets);
     sp.work_start = at<int32_t>(ws, pl.work_start); sp.totals = at<int32_t>(ws, pl.totals);
-    EXFOLD_CUDA(launch_prefill_sort(sp, s));
+    { ProfScope ps(1, s); EXFOLD_CUDA(launch_prefill_sort(sp, s)); }
 
     PrefillScatterParams cp{};
     cp.T = T; cp.N = N; cp.n_shared = l.n_shared; cp.Kp = Kp; cp.d_bytes = bf16 ? d * 2 : 0;
@@ -251,7 +306,7 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     cp.x = x; cp.xs = bf16 ? at<char>(ws, pl.xs) : nullptr;
     cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
     cp.row_w = at<float>(ws, pl.row_w); cp.row_exp = at<int32_t>(ws, pl.row_exp);
-    EXFOLD_CUDA(launch_prefill_scatter(cp, s));
+    { ProfScope ps(2, s); EXFOLD_CUDA(launch_prefill_scatter(cp, s)); }
 
     if (bf16) {
         if (!direct) EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.y32), 0, (size_t)T * d * 4, s));
@@ -263,19 +318,19 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
         g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
         const int64_t max_tiles = Rtot / kTileM + G;
         int grid1 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
-        EXFOLD_CUDA(launch_grouped_gemm1(g, grid1, s));
+        { ProfScope ps(3, s); EXFOLD_CUDA(launch_grouped_gemm1(g, grid1, s)); }
         g.tm_a = tm_h; g.tm_b0 = tm_wd; g.n_ntiles = (d + 255) / 256;
         g.y32 = direct ? nullptr : at<float>(ws, pl.y32);
         g.y = reinterpret_cast<__nv_bfloat16*>(y);
         int grid2 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
-        EXFOLD_CUDA(launch_grouped_gemm2(g, grid2, s));
-        if (!direct) EXFOLD_CUDA(launch_convert_bf16(at<float>(ws, pl.y32), T * d, y, s));
+        { ProfScope ps(4, s); EXFOLD_CUDA(launch_grouped_gemm2(g, grid2, s)); }
+        if (!direct) { ProfScope ps(5, s); EXFOLD_CUDA(launch_convert_bf16(at<float>(ws, pl.y32), T * d, y, s)); }
     } else {
         SimtFfnParams fp{};
         fp.x = x; fp.wg = w_gate; fp.wu = w_up; fp.wd = w_down; fp.dtype = l.dtype; fp.d = d; fp.I = I;
         fp.T = T; fp.Kr = Kp; fp.n_shared = l.n_shared; fp.N = N; fp.ids = rp.ids; fp.out = at<float>(ws, pl.out);
-        EXFOLD_CUDA(launch_simt_ffn(fp, s));
-        EXFOLD_CUDA(launch_combine_routes(fp.out, rp.w, T, Kp, d, l.n_shared, y, l.dtype, s));
+        { ProfScope ps(10, s); EXFOLD_CUDA(launch_simt_ffn(fp, s)); }
+        { ProfScope ps(11, s); EXFOLD_CUDA(launch_combine_routes(fp.out, rp.w, T, Kp, d, l.n_shared, y, l.dtype, s)); }
     }
     if (meta) {
         if ((rc = copy_meta(meta->ids, rp.ids, (size_t)R * 4, s))) return rc;
@@ -314,6 +369,7 @@ int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* log
                   make_tmap(&tm_wd, w_down, E * d, I, 128);
         if (!ok) return EXFOLD_ERR_CUDA;
     }
+    prof_reset();
     EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
 
     DecodeRouteParams rp{};
@@ -325,11 +381,11 @@ int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* log
     rp.row_tok = at<int32_t>(ws, pl.row_tok); rp.row_w = at<float>(ws, pl.row_w);
     rp.grp_expert = at<int32_t>(ws, pl.grp_expert); rp.grp_off = at<int32_t>(ws, pl.grp_off);
     rp.n_groups = at<int32_t>(ws, pl.n_groups);
-    EXFOLD_CUDA(launch_decode_route(rp, s));
+    { ProfScope ps(6, s); EXFOLD_CUDA(launch_decode_route(rp, s)); }
 
     if (bf16) {
-        EXFOLD_CUDA(launch_gather_rows(x, rp.row_tok, rp.n_groups + 1, max_rows, d * 2, at<char>(ws, pl.xs),
-                                       at<float>(ws, pl.y32), (int)B, d, s));
+        { ProfScope ps(7, s); EXFOLD_CUDA(launch_gather_rows(x, rp.row_tok, rp.n_groups + 1, max_rows, d * 2, at<char>(ws, pl.xs),
+                                       at<float>(ws, pl.y32), (int)B, d, s)); }
         DecodeFfnParams f{};
         f.tm_w0 = tm_wg; f.tm_w1 = tm_wu; f.tm_act = tm_xs;
         f.grp_expert = rp.grp_expert; f.grp_off = rp.grp_off; f.n_groups = rp.n_groups;
@@ -338,7 +394,7 @@ int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* log
         f.H = at<__nv_bfloat16>(ws, pl.H); f.y32 = at<float>(ws, pl.y32); f.status = at<DeviceStatus>(ws, pl.status);
         const int sms = sm_count();
         int items1 = f.max_groups * ((I + 127) / 128);
-        EXFOLD_CUDA(launch_decode_gateup(f, std::min(sms, items1), s));
+        { ProfScope ps(8, s); EXFOLD_CUDA(launch_decode_gateup(f, std::min(sms, items1), s)); }
         f.tm_w0 = tm_wd; f.tm_act = tm_h;
         const int n_ds = (d + 127) / 128, nkb = I / 64;
         int ks = (2 * sms + f.max_groups * n_ds - 1) / (f.max_groups * n_ds);
@@ -346,14 +402,14 @@ int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* log
         if (ks < 1) ks = 1;
         f.ksplit = ks;
         int items2 = f.max_groups * n_ds * ks;
-        EXFOLD_CUDA(launch_decode_down(f, std::min(sms, items2), s));
-        EXFOLD_CUDA(launch_convert_bf16(at<float>(ws, pl.y32), B * d, y, s));
+        { ProfScope ps(9, s); EXFOLD_CUDA(launch_decode_down(f, std::min(sms, items2), s)); }
+        { ProfScope ps(5, s); EXFOLD_CUDA(launch_convert_bf16(at<float>(ws, pl.y32), B * d, y, s)); }
     } else {
         SimtFfnParams fp{};
         fp.x = x; fp.wg = w_gate; fp.wu = w_up; fp.wd = w_down; fp.dtype = l.dtype; fp.d = d; fp.I = I;
         fp.T = B; fp.Kr = K; fp.n_shared = l.n_shared; fp.N = N; fp.ids = rp.ids; fp.out = at<float>(ws, pl.out);
-        EXFOLD_CUDA(launch_simt_ffn(fp, s));
-        EXFOLD_CUDA(launch_combine_routes(fp.out, rp.w, B, K, d, l.n_shared, y, l.dtype, s));
+        { ProfScope ps(10, s); EXFOLD_CUDA(launch_simt_ffn(fp, s)); }
+        { ProfScope ps(11, s); EXFOLD_CUDA(launch_combine_routes(fp.out, rp.w, B, K, d, l.n_shared, y, l.dtype, s)); }
     }
     if (meta) {
         if ((rc = copy_meta(meta->pool_ids, rp.pool_ids, (size_t)pool_m * 4, s))) return rc;
