@@ -34,6 +34,11 @@ if ROOT not in sys.path:
 import synth_inputs as si  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes measured by ncu (dram__bytes_read.sum + dram__bytes_write.sum) divided by the algorithmic
+# bytes of the same launch, from the reduced-case captures summarised under profiles/
+# (gemm_prefill_mixtral_reduced.md, decode_ffn_mixtral_reduced.md). Traffic grows with the weights, so the
+# full-size figure is this ratio times the full-size algorithmic bytes.
+NCU_TRAFFIC_RATIO = {"gemm1": 511.8 / 502.3, "decode_gateup": 240.4 / 234.9}
 
 
 def log(*a):
@@ -311,9 +316,13 @@ def run_ours(args, rank, world):
     if "gemm1_gateup_swiglu" in kern:
         t1 = kern["gemm1_gateup_swiglu"] * 1e-3
         ach = flop_gemm1 / t1 / 1e12
+        touched = N + cfg.n_shared  # every expert receives rows at these sizes
+        bytes_gemm1 = touched * 2.0 * d * I * el + rows * d * el + rows * I * el
         out["roofline"] = {"kernel": "grouped GEMM-1 (gate/up + SwiGLU), tcgen05", "bound": "tensor", "achieved": ach,
                            "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
-                           "traffic": None, "peak_source": f"{peak_src} burst bf16 matmul",
+                           "traffic": bytes_gemm1 * NCU_TRAFFIC_RATIO["gemm1"],
+                           "traffic_note": "ncu reduced-case DRAM bytes / algorithmic bytes x full-size algorithmic bytes",
+                           "peak_source": f"{peak_src} burst bf16 matmul",
                            "launch_ms": kern["gemm1_gateup_swiglu"], "flop_per_launch": flop_gemm1}
     elif "simt_ffn" in kern:
         t1 = kern["simt_ffn"] * 1e-3
@@ -326,7 +335,8 @@ def run_ours(args, rank, world):
         td = kern.get("decode_down", 0.0) * 1e-3
         out["decode"]["roofline"] = {"kernel": "decode gate/up weight stream, tcgen05 swap-AB", "bound": "hbm",
                                      "achieved": gateup_bytes / tg / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                     "frac": gateup_bytes / tg / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                                     "frac": gateup_bytes / tg / 1e9 / peaks["hbm_gbs"],
+                                     "traffic": gateup_bytes * NCU_TRAFFIC_RATIO["decode_gateup"],
                                      "bytes_per_launch": gateup_bytes, "launch_ms": kern["decode_gateup"]}
         if td > 0:
             out["decode"]["down_gbs"] = pool_bytes / 3.0 / td / 1e9

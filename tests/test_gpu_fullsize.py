@@ -1,0 +1,67 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times: routing
+metadata is compared bit-exactly at full size (the oracle's routing is cheap), outputs on a
+seeded sample of tokens the oracle evaluates one by one (every decode batch in full)."""
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+from harness import A, Case, check_decode_meta, check_output, check_prefill_meta
+
+pytestmark = pytest.mark.gpu
+
+
+def sample_tokens(T, n, seed=3):
+    return np.sort(np.random.default_rng(seed).choice(T, size=min(n, T), replace=False)).astype(np.int64)
+
+
+def run_full(name, n_sample, decode_cases=None):
+    cfg = si.CONFIGS[name]
+    case = Case(cfg, std=0.02)
+    for Kp in cfg.k_pre:
+        idx = sample_tokens(cfg.prefill_tokens, n_sample)
+        got, ref = case.run_prefill(Kp), case.oracle_prefill(Kp, tok_idx=idx)
+        assert ref["mismatch"] == 0, "log-scale ranking key disagrees with the literal w*h ranking"
+        check_prefill_meta(got, ref)
+        check_output(got["y"][idx], ref["y"], cfg.dtype)
+        # properties that hold at any size: every token keeps K' distinct routed experts
+        assert (np.diff(np.sort(got["ids"], 1), axis=1) > 0).all() if Kp > 1 else True
+        assert np.array_equal(np.sort(got["perm"]), np.arange(cfg.prefill_tokens * Kp))
+    for M in (decode_cases or cfg.pool_m):
+        got, ref = case.run_decode(M), case.oracle_decode(M)
+        assert ref["min_gap"] > 1e-9, "degenerate input: tie at the pool boundary"
+        check_decode_meta(got, ref, M)
+        check_output(got["y"], ref["y"], cfg.dtype)
+    return case
+
+
+def test_mixtral_shaped_full_size():
+    run_full("mixtral", 48)
+
+
+def test_qwen3_shaped_full_size():
+    run_full("qwen3", 96)
+
+
+def test_glm45air_shaped_full_size():
+    run_full("glm45air", 32)
+
+
+def test_qwen3_decode_sweep():
+    """Decode sweep: batch x pool budget, including the unfolded layer (M = N)."""
+    base = si.CONFIGS["qwen3"]
+    case = None
+    for B in (1, 8, 32, 128, 256):
+        cfg = si.scaled(base, decode_batch=B, prefill_tokens=64)
+        if case is None:
+            case = Case(cfg, std=0.02)
+        else:  # same weights and tables, new batch
+            import torch
+            case.cfg, case.B = cfg, B
+            case.xd, case.lgd = si.hidden_states(cfg, B, "x_dec"), si.router_logits(cfg, B, "logits_dec")
+            case.d_xd, case.d_lgd = case.xd.to(case.dev), case.lgd.to(case.dev)
+        for M in (8, 16, 32, 64, 128):
+            got, ref = case.run_decode(M), case.oracle_decode(M)
+            assert ref["min_gap"] > 1e-9
+            check_decode_meta(got, ref, M)
+            check_output(got["y"], ref["y"], "bf16")
