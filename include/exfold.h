@@ -48,6 +48,7 @@ enum {
     EXFOLD_ERR_WORKSPACE_TOO_SMALL = -3,
     EXFOLD_ERR_CUDA = -4,
     EXFOLD_ERR_DEVICE_TIMEOUT = -5,
+    EXFOLD_ERR_EXCEEDS_STATIC_SCRATCH = -6,
     EXFOLD_WARN_UNOBSERVED_EXPERT = 1
 };
 
@@ -167,6 +168,35 @@ int exfold_moe_decode_host(const exfold_layer *layer, const void *x_host, const 
                            int64_t B, const void *w_gate, const void *w_up, const void *w_down,
                            const exfold_tables *tables, int32_t pool_m, void *y_host,
                            const exfold_decode_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Decode for callers that cannot allocate device memory. (The paper has no counterpart: this is
+ * a packaging variant of exfold_moe_decode, same arguments minus the workspace, same results.)
+ *
+ * Who needs it: a host that must not call cudaMalloc while it runs - an engine whose memory pool
+ * is fixed at start-up, a plugin living in a process whose allocator it does not own, a caller
+ * that has already entered a phase where allocations are refused. Such a caller has nowhere to
+ * get the workspace from, so here the scratch is a fixed array of EXFOLD_STATIC_SCRATCH_BYTES
+ * inside the library image. Every GPU that loads the library holds those bytes until the process
+ * ends. The caller still passes inputs, outputs and optional metadata buffers as device pointers.
+ *
+ * Limits and rules:
+ *   - the call needs exfold_workspace_bytes(layer, B, layer->top_k) bytes; if that exceeds
+ *     EXFOLD_STATIC_SCRATCH_BYTES it returns EXFOLD_ERR_EXCEEDS_STATIC_SCRATCH and launches nothing
+ *     (e.g. Qwen3- and Mixtral-shaped layers fit up to B = 64, the GLM-4.5-Air-shaped one up to B = 32);
+ *   - it calls no cudaMalloc, cudaFree or any allocating library routine;
+ *   - the first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture;
+ *   - all calls on a device share the one array, which keeps what the previous call left in it;
+ *     the call itself clears what must start at zero, but two calls that overlap on the GPU
+ *     (different streams, no ordering between them) race on it: keep them on one stream or order
+ *     them with events.
+ */
+#define EXFOLD_STATIC_SCRATCH_BYTES (8u << 20)
+int exfold_moe_decode_noalloc(const exfold_layer *layer, const void *x, const float *logits, int64_t B,
+                              const void *w_gate, const void *w_up, const void *w_down,
+                              const exfold_tables *tables, int32_t pool_m, void *y,
+                              const exfold_decode_meta *meta, void *cuda_stream);
 
 /*
  * Synchronises the stream and decodes the status word the kernels keep at the start of the

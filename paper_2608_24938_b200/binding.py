@@ -22,11 +22,14 @@ EXFOLD_ERR_UNSUPPORTED = -2
 EXFOLD_ERR_WORKSPACE_TOO_SMALL = -3
 EXFOLD_ERR_CUDA = -4
 EXFOLD_ERR_DEVICE_TIMEOUT = -5
+EXFOLD_ERR_EXCEEDS_STATIC_SCRATCH = -6
+EXFOLD_STATIC_SCRATCH_BYTES = 8 << 20
 EXFOLD_WARN_UNOBSERVED_EXPERT = 1
 
 EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibrate", "exfold_moe_prefill",
            "exfold_moe_decode", "exfold_moe_prefill_host", "exfold_moe_decode_host", "exfold_device_status",
-           "exfold_status_string", "exfold_launch_count", "exfold_profile_enable", "exfold_profile_read"]
+           "exfold_status_string", "exfold_launch_count", "exfold_profile_enable", "exfold_profile_read",
+           "exfold_moe_decode_noalloc"]
 PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
                  "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
                  "simt_combine"]
@@ -77,6 +80,9 @@ def _load() -> C.CDLL:
         fn.restype = C.c_int
         fn.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables), i32, vp,
                        C.POINTER(exfold_decode_meta), vp, sz, vp]
+    lib.exfold_moe_decode_noalloc.restype = C.c_int
+    lib.exfold_moe_decode_noalloc.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables),
+                                              i32, vp, C.POINTER(exfold_decode_meta), vp]
     lib.exfold_device_status.restype = C.c_int
     lib.exfold_device_status.argtypes = [vp, vp]
     lib.exfold_status_string.restype = C.c_char_p
@@ -230,4 +236,18 @@ def exfold_moe_decode_host(layer, x_host, logits_host, w_gate, w_up, w_down, tab
                                     _decode_meta(meta), _ptr(ws), ws.numel(), _stream(stream))
     if check and rc != 0:
         raise ExfoldError(rc, "exfold_moe_decode_host")
+    return rc
+
+
+def exfold_moe_decode_noalloc(layer, x, logits, w_gate, w_up, w_down, tables: exfold_tables, pool_m: int, y,
+                              meta: Optional[dict] = None, stream=None, check: bool = True) -> int:
+    """Decode without a caller workspace, for hosts that may not allocate device memory: the scratch is
+    the library's own fixed array (EXFOLD_STATIC_SCRATCH_BYTES per GPU). Same results as
+    exfold_moe_decode. Calls on one device share that array, so keep them ordered on one stream; make
+    the first call on a device outside any stream capture."""
+    rc = lib.exfold_moe_decode_noalloc(C.byref(layer), _ptr(x), _ptr(logits), x.shape[0], _ptr(w_gate), _ptr(w_up),
+                                       _ptr(w_down), C.byref(tables), pool_m, _ptr(y), _decode_meta(meta),
+                                       _stream(stream))
+    if check and rc != 0:
+        raise ExfoldError(rc, "exfold_moe_decode_noalloc")
     return rc

@@ -240,6 +240,8 @@ const char* exfold_status_string(int status) {
         case EXFOLD_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case EXFOLD_ERR_CUDA: return "CUDA error";
         case EXFOLD_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+        case EXFOLD_ERR_EXCEEDS_STATIC_SCRATCH:
+            return "layer and batch need more scratch than the built-in EXFOLD_STATIC_SCRATCH_BYTES array holds";
         case EXFOLD_WARN_UNOBSERVED_EXPERT: return "warning: an expert was never observed during calibration";
         default: return "unknown status";
     }
