@@ -181,9 +181,10 @@ int exfold_moe_decode_host(const exfold_layer *layer, const void *x_host, const 
  * ends. The caller still passes inputs, outputs and optional metadata buffers as device pointers.
  *
  * Limits and rules:
- *   - the call needs exfold_workspace_bytes(layer, B, layer->top_k) bytes; if that exceeds
- *     EXFOLD_STATIC_SCRATCH_BYTES it returns EXFOLD_ERR_EXCEEDS_STATIC_SCRATCH and launches nothing
- *     (e.g. Qwen3- and Mixtral-shaped layers fit up to B = 64, the GLM-4.5-Air-shaped one up to B = 32);
+ *   - the call needs exfold_workspace_bytes(layer, B, layer->top_k) bytes of scratch; if that
+ *     exceeds EXFOLD_STATIC_SCRATCH_BYTES it returns EXFOLD_ERR_EXCEEDS_STATIC_SCRATCH and launches
+ *     nothing (e.g. Qwen3- and Mixtral-shaped layers fit up to B = 64, the GLM-4.5-Air-shaped
+ *     one up to B = 32);
  *   - it calls no cudaMalloc, cudaFree or any allocating library routine;
  *   - the first call on each device looks up the array's device address (with that device
  *     current); make that first call outside any stream capture;
@@ -219,7 +220,7 @@ int64_t exfold_launch_count(void);
  * each slot < n_slots, the elapsed milliseconds (or -1 if that kernel did not run in the last
  * call). Slots: 0 prefill route/fold, 1 prefill scan, 2 prefill scatter+gather, 3 grouped GEMM-1
  * (gate/up + SwiGLU), 4 grouped GEMM-2 (down + scatter-combine), 5 fp32->bf16 conversion,
- * 6 decode pool/remap, 7 decode row gather, 8 decode gate/up stream, 9 decode down stream,
+ * 6 decode pool/remap, 7 decode row gather, 8 decode GEMM-1 (gate/up stream), 9 decode GEMM-2 (down stream),
  * 10 SIMT expert FFN, 11 SIMT combine. Returns EXFOLD_OK or EXFOLD_ERR_CUDA.
  */
 #define EXFOLD_PROFILE_SLOTS 12

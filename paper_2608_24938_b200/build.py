@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libexfold.so")
 SOURCES = ["api.cu", "route_prefill.cu", "route_decode.cu", "ffn_simt.cu", "calibrate.cu", "gemm_prefill.cu",
-           "ffn_decode.cu", "no_alloc.cu"]
+           "no_alloc.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
 
@@ -28,12 +28,14 @@ def _newest_source_mtime() -> float:
     return max(os.path.getmtime(f) for f in files)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, extra_flags=(), lib_path: str = LIB, obj_dir: str = OBJ) -> str:
+    """extra_flags / lib_path / obj_dir let a debug variant (e.g. -DEXFOLD_TRACE) be built beside the product."""
     sources = list(SOURCES)
+    LIB, OBJ = lib_path, obj_dir  # noqa: N806
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source_mtime():
         return LIB
     os.makedirs(OBJ, exist_ok=True)
-    flags = list(FLAGS)
+    flags = list(FLAGS) + list(extra_flags)
     if verbose:
         flags = flags + ["-Xptxas", "-v"]
 
@@ -50,7 +52,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     with ThreadPoolExecutor(max(1, min(len(sources), os.cpu_count() or 1))) as ex:
         objs = list(ex.map(compile_one, sources))
     tmp = LIB + f".{os.getpid()}.tmp"
-    r = subprocess.run([NVCC, "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a"],
+    rdc = ["-rdc=true"] if "-rdc=true" in flags else []
+    r = subprocess.run([NVCC, "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a", *rdc],
                        capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")

@@ -1,15 +1,30 @@
 // C ABI of the folded-MoE library: argument validation, workspace planning, TMA tensor maps
 // and the launch sequences of the three calls. No device memory is allocated here.
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstring>
 
 #include "common.cuh"
+#include "ptx.cuh"
+
+#ifdef EXFOLD_TRACE
+namespace exfold {
+__device__ unsigned long long g_trace[4][kMaxCtas][kTraceSlots];
+}
+extern "C" int exfold_debug_read_trace(unsigned long long* out) {  // [4][kMaxCtas][kTraceSlots]
+    cudaDeviceSynchronize();
+    return cudaMemcpyFromSymbol(out, exfold::g_trace, sizeof(exfold::g_trace)) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 namespace exfold {
 
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+static thread_local bool t_pdl = false;
+void set_pdl(bool on) { t_pdl = on; }
+bool pdl_enabled() { return t_pdl; }
 
 namespace {
 
@@ -42,7 +57,7 @@ void prof_reset() {
 struct Plan {
     size_t status, ids, w, omit_src, omit_tgt, block_hist, offsets, work_start, totals, perm, row_tok, row_w,
         row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
-        xs, H, y32, out, total;
+        xs, H, y32, out, grp_tiles, total;
 };
 
 bool valid_layer(const exfold_layer* l) {
@@ -88,6 +103,7 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
     p.scale = take((size_t)N * 4);
     p.grp_expert = take((G + 2) * 4);
     p.grp_off = take((G + 2) * 4);
+    p.grp_tiles = take((G + 2) * 4);
     p.n_groups = take(16);
     p.zeros = take((size_t)N * 4);
     p.calib = take((size_t)N * N * (3 * 8 + 4) + (size_t)N * (8 + 4) + 256);
@@ -285,7 +301,6 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     }
 
     prof_reset();
-    EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
 
     PrefillRouteParams rp{};
     rp.logits = logits; rp.S = tables->S; rp.L = tables->L; rp.lnh = tables->lnh;
@@ -293,6 +308,7 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     rp.ids = at<int32_t>(ws, pl.ids); rp.w = at<float>(ws, pl.w);
     rp.omit_src = at<int32_t>(ws, pl.omit_src); rp.omit_tgt = at<int32_t>(ws, pl.omit_tgt);
     rp.block_hist = at<int32_t>(ws, pl.block_hist);
+    rp.status = at<DeviceStatus>(ws, pl.status);  // the first kernel of the call clears the status record
     { ProfScope ps(0, s); EXFOLD_CUDA(launch_prefill_route(rp, s)); }
 
     const int nblk = (int)((T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
@@ -308,14 +324,14 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     cp.x = x; cp.xs = bf16 ? at<char>(ws, pl.xs) : nullptr;
     cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
     cp.row_w = at<float>(ws, pl.row_w); cp.row_exp = at<int32_t>(ws, pl.row_exp);
+    cp.y32 = (bf16 && !direct) ? at<float>(ws, pl.y32) : nullptr; cp.d = d;
     { ProfScope ps(2, s); EXFOLD_CUDA(launch_prefill_scatter(cp, s)); }
 
     if (bf16) {
-        if (!direct) EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.y32), 0, (size_t)T * d * 4, s));
         GroupedGemmParams g{};
         g.tm_a = tm_xs; g.tm_a2 = tm_x; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu;
         g.offsets = sp.offsets; g.work_start = sp.work_start; g.G = G; g.n_routed = N; g.R = (int)R;
-        g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128;
+        g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.grp_expert = nullptr; g.n_groups_dev = nullptr;
         g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = cp.row_tok; g.row_w = cp.row_w;
         g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
         const int64_t max_tiles = Rtot / kTileM + G;
@@ -359,20 +375,21 @@ int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* log
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
     const bool bf16 = l.dtype == EXFOLD_BF16;
     const int max_rows = (int)(B * K + B * l.n_shared);
-    int NB = (int)((B + 15) / 16 * 16);
-    if (NB < 16) NB = 16;
 
     CUtensorMap tm_xs, tm_wg, tm_wu, tm_h, tm_wd;
     if (bf16) {
         const uint64_t E = (uint64_t)G;
-        bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)max_rows, d, NB) &&
+        bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)max_rows, d, 128) &&
                   make_tmap(&tm_wg, w_gate, E * I, d, 128) && make_tmap(&tm_wu, w_up, E * I, d, 128) &&
-                  make_tmap(&tm_h, at<char>(ws, pl.H), (uint64_t)max_rows, I, NB) &&
-                  make_tmap(&tm_wd, w_down, E * d, I, 128);
+                  make_tmap(&tm_h, at<char>(ws, pl.H), (uint64_t)max_rows, I, 128) &&
+                  make_tmap(&tm_wd, w_down, E * d, I, 256);
         if (!ok) return EXFOLD_ERR_CUDA;
     }
     prof_reset();
-    EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
+    struct PdlScope {
+        PdlScope() { set_pdl(true); }
+        ~PdlScope() { set_pdl(false); }
+    } pdl_scope;
 
     DecodeRouteParams rp{};
     rp.logits = logits; rp.S = tables->S; rp.L = tables->L; rp.h = tables->h;
@@ -382,29 +399,38 @@ int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* log
     rp.target = at<int32_t>(ws, pl.target); rp.scale = at<float>(ws, pl.scale);
     rp.row_tok = at<int32_t>(ws, pl.row_tok); rp.row_w = at<float>(ws, pl.row_w);
     rp.grp_expert = at<int32_t>(ws, pl.grp_expert); rp.grp_off = at<int32_t>(ws, pl.grp_off);
-    rp.n_groups = at<int32_t>(ws, pl.n_groups);
+    rp.grp_tiles = at<int32_t>(ws, pl.grp_tiles); rp.n_groups = at<int32_t>(ws, pl.n_groups);
+    rp.status = at<DeviceStatus>(ws, pl.status);
     { ProfScope ps(6, s); EXFOLD_CUDA(launch_decode_route(rp, s)); }
 
     if (bf16) {
         { ProfScope ps(7, s); EXFOLD_CUDA(launch_gather_rows(x, rp.row_tok, rp.n_groups + 1, max_rows, d * 2, at<char>(ws, pl.xs),
                                        at<float>(ws, pl.y32), (int)B, d, s)); }
-        DecodeFfnParams f{};
-        f.tm_w0 = tm_wg; f.tm_w1 = tm_wu; f.tm_act = tm_xs;
-        f.grp_expert = rp.grp_expert; f.grp_off = rp.grp_off; f.n_groups = rp.n_groups;
-        f.row_tok = rp.row_tok; f.row_w = rp.row_w; f.d = d; f.I = I; f.NB = NB; f.ksplit = 1;
-        f.max_groups = std::min(pool_m, N) + l.n_shared;
-        f.H = at<__nv_bfloat16>(ws, pl.H); f.y32 = at<float>(ws, pl.y32); f.status = at<DeviceStatus>(ws, pl.status);
-        const int sms = sm_count();
-        int items1 = f.max_groups * ((I + 127) / 128);
-        { ProfScope ps(8, s); EXFOLD_CUDA(launch_decode_gateup(f, std::min(sms, items1), s)); }
-        f.tm_w0 = tm_wd; f.tm_act = tm_h;
-        const int n_ds = (d + 127) / 128, nkb = I / 64;
-        int ks = (2 * sms + f.max_groups * n_ds - 1) / (f.max_groups * n_ds);
-        if (ks > nkb / 4) ks = nkb / 4;
-        if (ks < 1) ks = 1;
-        f.ksplit = ks;
-        int items2 = f.max_groups * n_ds * ks;
-        { ProfScope ps(9, s); EXFOLD_CUDA(launch_decode_down(f, std::min(sms, items2), s)); }
+        // The pool's rows (one per distinct (token, pool expert), grouped by pool rank) go through the
+        // same grouped GEMMs as prefill: tokens are the 128-row M operand (mostly padding, which costs
+        // nothing while the kernels are HBM-bound) and every MMA consumes 256 weight rows.
+        const int max_groups = std::min(pool_m, N) + l.n_shared;
+        const int tiles_per_group = (int)((B + kTileM - 1) / kTileM);
+        const int sms = std::min(sm_count(), kMaxCtas);
+        GroupedGemmParams g{};
+        g.tm_a = tm_xs; g.tm_a2 = tm_xs; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu;
+        g.offsets = rp.grp_off; g.work_start = rp.grp_tiles; g.G = max_groups; g.n_routed = 0x7fffffff;
+        g.R = max_rows; g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1;
+        g.grp_expert = rp.grp_expert; g.n_groups_dev = rp.n_groups;
+        g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = rp.row_tok; g.row_w = rp.row_w;
+        g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
+        const int64_t items1 = (int64_t)max_groups * tiles_per_group * g.n_ntiles;
+        { ProfScope ps(8, s); EXFOLD_CUDA(launch_grouped_gemm1(g, (int)std::min<int64_t>(sms, items1), s)); }
+        g.tm_a = tm_h; g.tm_b0 = tm_wd; g.n_ntiles = (d + 255) / 256;
+        g.y32 = at<float>(ws, pl.y32); g.y = reinterpret_cast<__nv_bfloat16*>(y);
+        // split K so that every SM streams a share of W_down even with few (expert, column tile) items
+        const int nkb2 = I / 64;
+        const int64_t base_items = (int64_t)max_groups * tiles_per_group * g.n_ntiles;
+        int ks = (int)((2 * (int64_t)sms + base_items - 1) / base_items);
+        ks = std::max(1, std::min(ks, nkb2 / 4));
+        const int kb_per = (nkb2 + ks - 1) / ks;
+        g.ksplit = (nkb2 + kb_per - 1) / kb_per;  // no empty parts
+        { ProfScope ps(9, s); EXFOLD_CUDA(launch_grouped_gemm2(g, (int)std::min<int64_t>(sms, base_items * g.ksplit), s)); }
         { ProfScope ps(5, s); EXFOLD_CUDA(launch_convert_bf16(at<float>(ws, pl.y32), B * d, y, s)); }
     } else {
         SimtFfnParams fp{};
@@ -453,6 +479,7 @@ int exfold_calibrate(const exfold_layer* layer, const void* x_cal, const float* 
         rp.logits = logits_cal; rp.S = out->S; rp.L = out->L; rp.lnh = at<float>(ws, pl.zeros);
         rp.T = m; rp.N = N; rp.K = K; rp.Kp = K; rp.ids = ids; rp.w = at<float>(ws, pl.w);
         rp.omit_src = nullptr; rp.omit_tgt = nullptr; rp.block_hist = at<int32_t>(ws, pl.block_hist);
+        rp.status = nullptr;
         EXFOLD_CUDA(launch_prefill_route(rp, s));
     } else {
         EXFOLD_CUDA(launch_iota_ids(ids, m, N, s));

@@ -23,6 +23,7 @@ constexpr int kMaxTopK = 32;
 constexpr int kMaxGroups = kMaxExperts + 1;  // + shared expert
 constexpr int kTileM = 128;                  // token rows per prefill GEMM tile
 constexpr int kMaxDecodeBatch = 256;
+constexpr int kMaxCtas = 160;                // persistent grids never exceed this (148 SMs on B200)
 
 __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
     if (atomicCAS(&st->code, 0, EXFOLD_ERR_DEVICE_TIMEOUT) == 0) {
@@ -33,6 +34,36 @@ __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
 
 // host-side launch accounting
 void count_launch(int n = 1);
+
+// Programmatic dependent launch: every kernel of the library is launched with the "programmatic stream
+// serialization" attribute, lets its successor be scheduled early (grid_dep_launch) and waits for its
+// predecessor's results (grid_dep_wait) before it touches global memory. This removes the several
+// microseconds of launch latency between dependent kernels of one call. Both are no-ops when the
+// kernel was launched without the attribute.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Programmatic launch is requested per call chain: it pays for the short, latency-bound decode chain and
+// measured slower for prefill (early-resident successors compete with the running kernel).
+void set_pdl(bool on);
+bool pdl_enabled();
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+    count_launch();
+    return e;
+}
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -49,6 +80,7 @@ struct PrefillRouteParams {
     int32_t* omit_src;  // [T][K-Kp] or null
     int32_t* omit_tgt;  // [T][K-Kp] or null
     int32_t* block_hist;  // [nblk][N]
+    DeviceStatus* status; // cleared by block 0 (first kernel of a call); may be null
 };
 constexpr int kRouteTokensPerBlock = 64;
 constexpr int kRouteThreads = 512;
@@ -75,6 +107,8 @@ struct PrefillScatterParams {
     int32_t* row_tok;   // [R + T*n_shared]
     float* row_w;       // [R + T*n_shared]
     int32_t* row_exp;   // [R + T*n_shared]
+    float* y32;         // fp32 accumulator [T][d] to clear (null: nothing to clear)
+    int d;
 };
 
 cudaError_t launch_prefill_route(const PrefillRouteParams& p, cudaStream_t s);
@@ -101,7 +135,9 @@ struct DecodeRouteParams {
     float* row_w;         // [B*K + B]
     int32_t* grp_expert;  // [N+1] expert id of each group (pool order; shared last)
     int32_t* grp_off;     // [N+2] first row of each group
+    int32_t* grp_tiles;   // [N+2] prefix of 128-row tiles per group (work list of the grouped GEMMs)
     int32_t* n_groups;    // [2]: number of groups, total rows
+    DeviceStatus* status; // cleared here (first kernel of a decode call)
 };
 cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s);
 cudaError_t launch_gather_rows(const void* x, const int32_t* row_tok, const int32_t* n_rows_ptr, int max_rows,
@@ -158,6 +194,9 @@ struct GroupedGemmParams {
     int R;                      // routed rows (shared rows start here)
     int d, I;
     int n_ntiles;               // column tiles
+    int ksplit;                 // GEMM-2: K parts per tile (> 1 only with the y32 reduction epilogue)
+    const int32_t* grp_expert;  // [G] expert whose weights group g uses (null: g itself)
+    const int32_t* n_groups_dev;  // device-side group count (null: G)
     // epilogues
     __nv_bfloat16* H;           // GEMM-1 out [Rtot][I]
     const int32_t* row_tok;     // GEMM-2
@@ -168,22 +207,5 @@ struct GroupedGemmParams {
 };
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s);
 cudaError_t launch_grouped_gemm2(const GroupedGemmParams& p, int grid, cudaStream_t s);
-
-struct DecodeFfnParams {
-    CUtensorMap tm_w0;  // gate/up kernel: W_gate [(E*I)][d]; down kernel: W_down [(E*d)][I]
-    CUtensorMap tm_w1;  // gate/up kernel: W_up
-    CUtensorMap tm_act; // gate/up kernel: Xs [rows][d]; down kernel: H [rows][I]; box rows = NB
-    const int32_t* grp_expert;
-    const int32_t* grp_off;
-    const int32_t* n_groups;
-    const int32_t* row_tok;
-    const float* row_w;
-    int d, I, NB, ksplit, max_groups;
-    __nv_bfloat16* H;  // [rows][I]
-    float* y32;        // [B][d]
-    DeviceStatus* status;
-};
-cudaError_t launch_decode_gateup(const DecodeFfnParams& p, int grid, cudaStream_t s);
-cudaError_t launch_decode_down(const DecodeFfnParams& p, int grid, cudaStream_t s);
 
 }  // namespace exfold

@@ -26,6 +26,8 @@ __global__ void __launch_bounds__(256) simt_ffn_kernel(SimtFfnParams p) {
     float* xs = sm;          // [d]
     float* act = sm + p.d;   // [I]
     const int64_t row = blockIdx.x;
+    grid_dep_launch();
+    grid_dep_wait();
     const int64_t n_routed = p.T * p.Kr;
     int64_t tok;
     int e;
@@ -71,6 +73,8 @@ template <typename T>
 __global__ void combine_routes_kernel(const float* __restrict__ out, const float* __restrict__ w, int64_t Tn,
                                       int Kr, int d, int n_shared, T* __restrict__ y) {
     const int64_t i = blockIdx.x;
+    grid_dep_launch();
+    grid_dep_wait();
     for (int c = threadIdx.x; c < d; c += blockDim.x) {
         float acc = 0.f;
         for (int j = 0; j < Kr; ++j) acc = fmaf(w[i * Kr + j], out[(size_t)(i * Kr + j) * d + c], acc);
@@ -83,6 +87,8 @@ __global__ void combine_routes_kernel(const float* __restrict__ out, const float
 __global__ void convert_bf16_kernel(const float4* __restrict__ src, int64_t n4, uint2* __restrict__ dst) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    grid_dep_launch();
+    grid_dep_wait();
     for (; i < n4; i += stride) {
         float4 v = src[i];
         __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y);
@@ -105,27 +111,22 @@ cudaError_t launch_simt_ffn(const SimtFfnParams& p, cudaStream_t s) {
         err = cudaFuncSetAttribute(simt_ffn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)smem);
         if (err != cudaSuccess) return err;
-        simt_ffn_kernel<__nv_bfloat16><<<(unsigned)rows, 256, smem, s>>>(p);
+        return launch_pdl(simt_ffn_kernel<__nv_bfloat16>, (unsigned)rows, 256, smem, s, p);
     } else {
         err = cudaFuncSetAttribute(simt_ffn_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
-        simt_ffn_kernel<float><<<(unsigned)rows, 256, smem, s>>>(p);
+        return launch_pdl(simt_ffn_kernel<float>, (unsigned)rows, 256, smem, s, p);
     }
-    count_launch();
-    return cudaGetLastError();
 }
 
 cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, int Kr, int d, int n_shared,
                                   void* y, int dtype, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
     if (dtype == EXFOLD_BF16)
-        combine_routes_kernel<__nv_bfloat16><<<(unsigned)T, 256, 0, s>>>(out, w, T, Kr, d, n_shared,
-                                                                         reinterpret_cast<__nv_bfloat16*>(y));
-    else
-        combine_routes_kernel<float><<<(unsigned)T, 256, 0, s>>>(out, w, T, Kr, d, n_shared,
-                                                                 reinterpret_cast<float*>(y));
-    count_launch();
-    return cudaGetLastError();
+        return launch_pdl(combine_routes_kernel<__nv_bfloat16>, (unsigned)T, 256, 0, s, out, w, T, Kr, d, n_shared,
+                          reinterpret_cast<__nv_bfloat16*>(y));
+    return launch_pdl(combine_routes_kernel<float>, (unsigned)T, 256, 0, s, out, w, T, Kr, d, n_shared,
+                      reinterpret_cast<float*>(y));
 }
 
 cudaError_t launch_convert_bf16(const float* y32, int64_t n, void* y, cudaStream_t s) {
@@ -133,10 +134,8 @@ cudaError_t launch_convert_bf16(const float* y32, int64_t n, void* y, cudaStream
     const int64_t n4 = n / 4;  // n is a multiple of 64 (d is)
     int blocks = (int)((n4 + 255) / 256);
     if (blocks > 148 * 16) blocks = 148 * 16;
-    convert_bf16_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(y32), n4,
-                                               reinterpret_cast<uint2*>(y));
-    count_launch();
-    return cudaGetLastError();
+    return launch_pdl(convert_bf16_kernel, blocks, 256, 0, s, reinterpret_cast<const float4*>(y32), n4,
+                      reinterpret_cast<uint2*>(y));
 }
 
 }  // namespace exfold

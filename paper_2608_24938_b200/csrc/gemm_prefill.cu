@@ -31,10 +31,13 @@ constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;
 
 struct WorkItem {
-    int g, row0, rows, n_idx;
+    int g, row0, rows, n_idx, kpart;
 };
 
-__device__ __forceinline__ WorkItem decode_work(int w, int G, int nt, const int* s_off, const int* s_ws) {
+// Work index -> (group, row tile, column tile, K part). Order: group, column tile, row tile, K part
+// (fastest), so CTAs running together share weight tiles through L2.
+__device__ __forceinline__ WorkItem decode_work(int w_all, int G, int nt, int ks, const int* s_off, const int* s_ws) {
+    const int w = ks == 1 ? w_all : w_all / ks;
     int lo = 0, hi = G;  // find g with s_ws[g]*nt <= w < s_ws[g+1]*nt
     while (hi - lo > 1) {
         int mid = (lo + hi) >> 1;
@@ -45,6 +48,7 @@ __device__ __forceinline__ WorkItem decode_work(int w, int G, int nt, const int*
     while (lo + 1 < G && s_ws[lo + 1] * nt <= w) ++lo;
     WorkItem it;
     it.g = lo;
+    it.kpart = w_all - w * ks;
     const int tiles = s_ws[lo + 1] - s_ws[lo];
     const int local = w - s_ws[lo] * nt;
     const int m_idx = local % tiles;
@@ -60,7 +64,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int MODE>  // 0: gate/up + SwiGLU -> H; 1: down + weighted scatter -> y
+// MODE 0: gate/up + SwiGLU -> H; MODE 1: down + weighted scatter -> y.
+// DEC (decode) adds what only the expert-pool path needs: a group -> expert map, a group count that is
+// known only on the device, and split-K for GEMM-2. The prefill instantiations compile all of it away.
+template <int MODE, bool DEC>
 __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __grid_constant__ GroupedGemmParams p) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kStages];
@@ -71,17 +78,25 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     __shared__ int abort_s;
     __shared__ int s_off[kMaxGroups + 1];
     __shared__ int s_ws[kMaxGroups + 1];
+    __shared__ int s_exp[kMaxGroups + 1];
 
     unsigned char* tiles =
         reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = p.G;
-
-    for (int i = threadIdx.x; i <= G; i += kGemmThreads) {
-        s_off[i] = p.offsets[i];
-        s_ws[i] = p.work_start[i];
-    }
+    constexpr int kTr = MODE;  // trace table of this kernel (debug builds only)
+    (void)kTr;
+    if (threadIdx.x == 0) EXFOLD_TRACE_SET(kTr, 0, ptx::globaltimer_ns());
+    long long tr_wait = 0, tr_wait2 = 0;
+    (void)tr_wait;
+    (void)tr_wait2;
+    // ---- prologue that does not depend on earlier kernels: overlaps their tail under programmatic launch
     if (threadIdx.x == 0) {
+        ptx::prefetch_tmap(&p.tm_a);
+        ptx::prefetch_tmap(&p.tm_b0);
+        if (MODE == 0) {
+            ptx::prefetch_tmap(&p.tm_a2);
+            ptx::prefetch_tmap(&p.tm_b1);
+        }
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(&full_bar[s], 1);
             ptx::mbar_init(&empty_bar[s], 1);
@@ -92,57 +107,76 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         }
         abort_s = 0;
         ptx::fence_mbar_init();
-        ptx::prefetch_tmap(&p.tm_a);
-        ptx::prefetch_tmap(&p.tm_b0);
-        if (MODE == 0) {
-            ptx::prefetch_tmap(&p.tm_a2);
-            ptx::prefetch_tmap(&p.tm_b1);
-        }
     }
     if (warp == 1) {
         ptx::tmem_alloc(&tmem_base_s, kTmemCols);
         ptx::tmem_relinquish();
+    }
+    grid_dep_wait();  // everything below reads what the routing kernels (or GEMM-1) wrote
+    int G = p.G;
+    if (DEC) {  // the number of groups (pool size) is known only on the device
+        const int gd = *p.n_groups_dev;
+        G = gd < G ? gd : G;
+    }
+    for (int i = threadIdx.x; i <= G; i += kGemmThreads) {
+        s_off[i] = p.offsets[i];
+        s_ws[i] = p.work_start[i];
+        if (DEC) s_exp[i] = i < G ? p.grp_expert[i] : i;  // group -> expert whose weights it uses
     }
     ptx::tc_fence_before();
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
     const int nt = p.n_ntiles;
-    const int total = s_ws[G] * nt;
+    const int ks = (DEC && MODE == 1) ? p.ksplit : 1;  // K parts per tile (needs the fp32-reduction epilogue)
+    const int total = s_ws[G] * nt * ks;
+    // Effective grid: with `rounds` items per CTA, ceil(total / rounds) CTAs finish together; the rest
+    // stay idle instead of leaving a few CTAs one item behind (448 items on 148 SMs: 112 x 4, not
+    // 144 x 3 + 4 x 4). A hundred SMs are enough to saturate HBM when the kernel is memory-bound.
+    const int rounds = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int eff_grid = rounds > 0 ? (total + rounds - 1) / rounds : 0;
+    const int w_begin = (int)blockIdx.x < eff_grid ? (int)blockIdx.x : total;  // idle CTAs see no work
+    const int w_stride = eff_grid > 0 ? eff_grid : 1;
     const int nkb = (MODE == 0 ? p.d : p.I) / kBK;
+    const int kb_per = (nkb + ks - 1) / ks;
     volatile int* abort_flag = &abort_s;
+    if (threadIdx.x == 0) EXFOLD_TRACE_SET(kTr, 1, ptx::globaltimer_ns());
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
             int stage = 0, phase = 0;
             bool ok = true;
-            for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-                const WorkItem it = decode_work(w, G, nt, s_off, s_ws);
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (!ptx::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, p.status, 1)) {
+            for (int w = w_begin; w < total && ok; w += w_stride) {
+                const WorkItem it = decode_work(w, G, nt, ks, s_off, s_ws);
+                const int kb0 = it.kpart * kb_per, kb1 = min(nkb, kb0 + kb_per);
+                // per-tile constants stay in registers: the k-loop below is the latency-critical path
+                const int expert = DEC ? s_exp[it.g] : it.g;
+                const bool from_x = !DEC && MODE == 0 && expert >= p.n_routed;  // prefill's shared expert reads x directly
+                const CUtensorMap* tma_a = from_x ? &p.tm_a2 : &p.tm_a;
+                const int arow = from_x ? it.row0 - p.R : it.row0;
+                const int brow = MODE == 0 ? expert * p.I + it.n_idx * 128 : expert * p.d + it.n_idx * 256;
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    bool got;
+                    EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, p.status, 1));
+                    if (!got) {
                         ok = false;
                         break;
                     }
                     unsigned char* a_dst = tiles + stage * kStageBytes;
                     unsigned char* b_dst = a_dst + kATileBytes;
                     ptx::mbar_expect_tx(&full_bar[stage], kStageBytes);
-                    if (MODE == 0) {
-                        if (it.g < p.n_routed) ptx::tma_load_2d(a_dst, &p.tm_a, &full_bar[stage], kb * kBK, it.row0);
-                        else ptx::tma_load_2d(a_dst, &p.tm_a2, &full_bar[stage], kb * kBK, it.row0 - p.R);
-                        const int brow = it.g * p.I + it.n_idx * 128;
-                        ptx::tma_load_2d(b_dst, &p.tm_b0, &full_bar[stage], kb * kBK, brow);
-                        ptx::tma_load_2d(b_dst + 128 * 128, &p.tm_b1, &full_bar[stage], kb * kBK, brow);
-                    } else {
-                        ptx::tma_load_2d(a_dst, &p.tm_a, &full_bar[stage], kb * kBK, it.row0);
-                        ptx::tma_load_2d(b_dst, &p.tm_b0, &full_bar[stage], kb * kBK, it.g * p.d + it.n_idx * 256);
-                    }
+                    ptx::tma_load_2d(a_dst, tma_a, &full_bar[stage], kb * kBK, arow);
+                    ptx::tma_load_2d(b_dst, &p.tm_b0, &full_bar[stage], kb * kBK, brow);
+                    if (MODE == 0) ptx::tma_load_2d(b_dst + 128 * 128, &p.tm_b1, &full_bar[stage], kb * kBK, brow);
                     if (++stage == kStages) {
                         stage = 0;
                         phase ^= 1;
                     }
                 }
             }
+            EXFOLD_TRACE_SET(kTr, 3, tr_wait);
+            EXFOLD_TRACE_SET(kTr, 4, ptx::globaltimer_ns());
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -151,13 +185,19 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
             constexpr uint32_t idesc = ptx::make_idesc_bf16(128, 256);
             int stage = 0, phase = 0, iter = 0;
             bool ok = true;
-            for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++iter) {
+            for (int w = w_begin; w < total && ok; w += w_stride, ++iter) {
                 const int as = iter & 1, aphase = (iter >> 1) & 1;
-                if (!ptx::mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag, p.status, 2)) break;
+                bool got;
+                EXFOLD_TRACE_ADD(tr_wait2, got = ptx::mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag, p.status, 2));
+                if (!got) break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + as * 256;
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (!ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3)) {
+                const int kpart = ks == 1 ? 0 : w % ks;
+                const int kb0 = kpart * kb_per, kb1 = min(nkb, kb0 + kb_per);
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3));
+                    if (iter == 0 && kb == kb0) EXFOLD_TRACE_SET(kTr, 9, ptx::globaltimer_ns());
+                    if (!got) {
                         ok = false;
                         break;
                     }
@@ -167,7 +207,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                     const uint64_t bdesc = ptx::make_kmajor_sw128_desc(a_addr + kATileBytes);
 #pragma unroll
                     for (int k = 0; k < kBK / 16; ++k)
-                        ptx::umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                        ptx::umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
                     ptx::umma_commit(&empty_bar[stage]);
                     if (++stage == kStages) {
                         stage = 0;
@@ -176,19 +216,31 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                 }
                 if (ok) ptx::umma_commit(&tfull_bar[as]);
             }
+            EXFOLD_TRACE_SET(kTr, 5, tr_wait);
+            EXFOLD_TRACE_SET(kTr, 6, tr_wait2);
+            EXFOLD_TRACE_SET(kTr, 7, ptx::globaltimer_ns());
+            EXFOLD_TRACE_SET(kTr, 10, iter);
         }
         __syncwarp();
     } else {
         // ------------------------------------------------ epilogue warps (TMEM lane quadrant = warp % 4)
         const int q = warp & 3;
         int iter = 0;
-        for (int w = blockIdx.x; w < total; w += gridDim.x, ++iter) {
+        for (int w = w_begin; w < total; w += w_stride, ++iter) {
             const int as = iter & 1, aphase = (iter >> 1) & 1;
-            const WorkItem it = decode_work(w, G, nt, s_off, s_ws);
-            if (!ptx::mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status, 4)) break;
+            const WorkItem it = decode_work(w, G, nt, ks, s_off, s_ws);
+            // lane 0 waits; the warp takes one decision, so the warp-wide TMEM loads below stay convergent
+            int ok = 1;
+            if (lane == 0) {
+                bool got;
+                EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status, 4));
+                ok = got ? 1 : 0;
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
             ptx::tc_fence_after();
             const int row = q * 32 + lane;
-            const bool valid = row < it.rows;
+            const bool valid = row < it.rows && it.kpart * kb_per < nkb;  // a K part without k-blocks adds nothing
             const int64_t grow = (int64_t)it.row0 + row;
             const uint32_t taddr = tmem_base + as * 256 + ((uint32_t)(q * 32) << 16);
             if (MODE == 0) {
@@ -256,6 +308,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     }
 
     // ------------------------------------------------ teardown
+    // Only now may the next kernel's CTAs be scheduled: released earlier they would sit on the SMs
+    // waiting for this grid and compete for issue slots with the few warps that drive the pipeline.
+    // One thread fires it, after the epilogue loop (a single call marks the whole CTA as triggered).
+    if (threadIdx.x == 64) {
+        grid_dep_launch();
+        EXFOLD_TRACE_SET(kTr, 8, tr_wait);
+        EXFOLD_TRACE_SET(kTr, 11, ptx::globaltimer_ns());
+    }
     ptx::tc_fence_before();
     __syncthreads();
     if (abort_s) __nanosleep(100000);  // let any copy still in flight land before shared memory is released
@@ -263,30 +323,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
+    if (threadIdx.x == 0) EXFOLD_TRACE_SET(kTr, 2, ptx::globaltimer_ns());
 }
 
 }  // namespace
 
-static cudaError_t launch_gemm(const GroupedGemmParams& p, int grid, cudaStream_t s, int mode) {
-    cudaError_t err;
-    if (mode == 0) {
-        err = cudaFuncSetAttribute(grouped_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
-        if (err != cudaSuccess) return err;
-        grouped_gemm_kernel<0><<<grid, kGemmThreads, kGemmSmem, s>>>(p);
-    } else {
-        err = cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
-        if (err != cudaSuccess) return err;
-        grouped_gemm_kernel<1><<<grid, kGemmThreads, kGemmSmem, s>>>(p);
-    }
-    count_launch();
-    return cudaGetLastError();
+template <int MODE, bool DEC>
+static cudaError_t launch_gemm_t(const GroupedGemmParams& p, int grid, cudaStream_t s) {
+    cudaError_t err = cudaFuncSetAttribute(grouped_gemm_kernel<MODE, DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           kGemmSmem);
+    if (err != cudaSuccess) return err;
+    return launch_pdl(grouped_gemm_kernel<MODE, DEC>, grid, kGemmThreads, kGemmSmem, s, p);
 }
 
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s) {
-    return launch_gemm(p, grid, s, 0);
+    return p.grp_expert != nullptr ? launch_gemm_t<0, true>(p, grid, s) : launch_gemm_t<0, false>(p, grid, s);
 }
 cudaError_t launch_grouped_gemm2(const GroupedGemmParams& p, int grid, cudaStream_t s) {
-    return launch_gemm(p, grid, s, 1);
+    return p.grp_expert != nullptr ? launch_gemm_t<1, true>(p, grid, s) : launch_gemm_t<1, false>(p, grid, s);
 }
 
 }  // namespace exfold

@@ -42,13 +42,12 @@ extern "C" int exfold_moe_decode_noalloc(const exfold_layer* layer, const void* 
                                          const exfold_tables* tables, int32_t pool_m, void* y,
                                          const exfold_decode_meta* meta, void* cuda_stream) {
     if (layer == nullptr || B < 1) return EXFOLD_ERR_INVALID_ARG;
-    const size_t need = exfold_workspace_bytes(layer, B, layer->top_k);
-    if (need == 0) return EXFOLD_ERR_INVALID_ARG;
-    if (need > (size_t)EXFOLD_STATIC_SCRATCH_BYTES) return EXFOLD_ERR_EXCEEDS_STATIC_SCRATCH;
     void* ws = scratch_for_current_device();
     if (ws == nullptr) return EXFOLD_ERR_CUDA;
-    // The ordinary call clears, on the stream, everything in the scratch that has to start at zero
-    // (the status record and the fp32 accumulator); the rest is overwritten before it is read.
-    return exfold_moe_decode(layer, x, logits, B, w_gate, w_up, w_down, tables, pool_m, y, meta, ws, need,
-                             cuda_stream);
+    // The ordinary call checks that the array is large enough before it launches anything, and clears,
+    // on the stream, everything in the scratch that has to start at zero (the status record and the
+    // fp32 accumulator); the rest is overwritten before it is read.
+    int rc = exfold_moe_decode(layer, x, logits, B, w_gate, w_up, w_down, tables, pool_m, y, meta, ws,
+                               (size_t)EXFOLD_STATIC_SCRATCH_BYTES, cuda_stream);
+    return rc == EXFOLD_ERR_WORKSPACE_TOO_SMALL ? EXFOLD_ERR_EXCEEDS_STATIC_SCRATCH : rc;
 }

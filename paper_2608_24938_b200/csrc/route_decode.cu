@@ -34,6 +34,9 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kDecThreads / 32;
     const int B = p.B, N = p.N, K = p.K, M = p.M;
+    grid_dep_launch();
+    grid_dep_wait();
+    if (p.status != nullptr && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
 
     // ---- Eq. 2 per token (warp per token), weights in double
     for (int i = warp; i < B; i += kWarps) {
@@ -230,6 +233,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         p.grp_off[g] = sm.goff[g];
         if (g < G) p.grp_expert[g] = g < P ? sm.pool[g] : N;
     }
+    if (threadIdx.x == 0) {  // prefix of 128-row tiles per group
+        int tiles = 0;
+        for (int g = 0; g < G; ++g) {
+            p.grp_tiles[g] = tiles;
+            tiles += (sm.goff[g + 1] - sm.goff[g] + kTileM - 1) / kTileM;
+        }
+        p.grp_tiles[G] = tiles;
+    }
     if (p.n_shared)
         for (int i = threadIdx.x; i < B; i += kDecThreads) {
             p.row_tok[sm.goff[P] + i] = i;
@@ -249,6 +260,8 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const void* __restrict
                                                           void* __restrict__ xs, float* __restrict__ y32,
                                                           int zero_rows, int zero_row_floats) {
     const int row = blockIdx.x;
+    grid_dep_launch();
+    grid_dep_wait();
     if (y32 != nullptr && row < zero_rows) {
         float4* z = reinterpret_cast<float4*>(y32 + (size_t)row * zero_row_floats);
         for (int c = threadIdx.x; c < zero_row_floats / 4; c += blockDim.x) z[c] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -270,7 +283,7 @@ cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s) {
     err = cudaFuncSetAttribute(decode_route_kernel<NPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
                                (int)smem);                                                                  \
     if (err != cudaSuccess) return err;                                                                     \
-    decode_route_kernel<NPL><<<1, kDecThreads, smem, s>>>(p);
+    err = launch_pdl(decode_route_kernel<NPL>, 1, kDecThreads, smem, s, p);
     switch (npl) {
         case 1: EXFOLD_DEC_LAUNCH(1) break;
         case 2: EXFOLD_DEC_LAUNCH(2) break;
@@ -278,8 +291,7 @@ cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s) {
         default: EXFOLD_DEC_LAUNCH(8) break;
     }
 #undef EXFOLD_DEC_LAUNCH
-    count_launch();
-    return cudaGetLastError();
+    return err;
 }
 
 cudaError_t launch_gather_rows(const void* x, const int32_t* row_tok, const int32_t* n_rows_ptr, int max_rows,
@@ -287,10 +299,8 @@ cudaError_t launch_gather_rows(const void* x, const int32_t* row_tok, const int3
                                cudaStream_t s) {
     int grid = max_rows > zero_rows ? max_rows : zero_rows;
     if (grid == 0) return cudaSuccess;
-    gather_rows_kernel<<<grid, 256, 0, s>>>(x, row_tok, n_rows_ptr, row_bytes, xs, y32, zero_rows,
-                                            zero_row_floats);
-    count_launch();
-    return cudaGetLastError();
+    return launch_pdl(gather_rows_kernel, grid, 256, 0, s, x, row_tok, n_rows_ptr, row_bytes, xs, y32, zero_rows,
+                      zero_row_floats);
 }
 
 }  // namespace exfold

@@ -21,8 +21,11 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_route_kernel(PrefillRou
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     constexpr int kWarps = kRouteThreads / 32;
+    grid_dep_launch();
     for (int e = threadIdx.x; e < p.N; e += blockDim.x) hist[e] = 0;
     __syncthreads();
+    grid_dep_wait();
+    if (p.status != nullptr && blockIdx.x == 0 && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
 
     const int N = p.N, K = p.K, Kp = p.Kp, Ko = p.K - p.Kp;
     const int64_t tok0 = (int64_t)blockIdx.x * kRouteTokensPerBlock;
@@ -128,6 +131,8 @@ __global__ void __launch_bounds__(1024) prefill_sort_kernel(PrefillSortParams p)
     __shared__ int tot[kMaxGroups + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int N = p.N;
+    grid_dep_launch();
+    grid_dep_wait();
     for (int e = warp; e < N; e += nwarps) {
         int run = 0;
         for (int b0 = 0; b0 < p.nblk; b0 += 32) {
@@ -171,6 +176,13 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_scatter_kernel(PrefillS
     const int ntok = (int)min((int64_t)kRouteTokensPerBlock, p.T - tok0);
     const int n = ntok * Kp;
     const int64_t r0 = tok0 * Kp;
+    grid_dep_launch();
+    grid_dep_wait();
+    if (p.y32 != nullptr) {  // clear this block's rows of the fp32 accumulator
+        float4* z = reinterpret_cast<float4*>(p.y32 + (size_t)tok0 * p.d);
+        const int n4 = ntok * p.d / 4;
+        for (int c = threadIdx.x; c < n4; c += blockDim.x) z[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     for (int e = threadIdx.x; e < N; e += blockDim.x)
         cnt[e] = p.offsets[e] + p.block_hist[(size_t)blockIdx.x * N + e];
     __syncthreads();
@@ -226,26 +238,20 @@ cudaError_t launch_prefill_route(const PrefillRouteParams& p, cudaStream_t s) {
     const int nblk = (int)((p.T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
     const int npl = (p.N + 31) / 32;
     switch (npl) {
-        case 1: prefill_route_kernel<1><<<nblk, kRouteThreads, 0, s>>>(p); break;
-        case 2: prefill_route_kernel<2><<<nblk, kRouteThreads, 0, s>>>(p); break;
-        case 3: case 4: prefill_route_kernel<4><<<nblk, kRouteThreads, 0, s>>>(p); break;
-        default: prefill_route_kernel<8><<<nblk, kRouteThreads, 0, s>>>(p); break;
+        case 1: return launch_pdl(prefill_route_kernel<1>, nblk, kRouteThreads, 0, s, p);
+        case 2: return launch_pdl(prefill_route_kernel<2>, nblk, kRouteThreads, 0, s, p);
+        case 3: case 4: return launch_pdl(prefill_route_kernel<4>, nblk, kRouteThreads, 0, s, p);
+        default: return launch_pdl(prefill_route_kernel<8>, nblk, kRouteThreads, 0, s, p);
     }
-    count_launch();
-    return cudaGetLastError();
 }
 
 cudaError_t launch_prefill_sort(const PrefillSortParams& p, cudaStream_t s) {
-    prefill_sort_kernel<<<1, 1024, 0, s>>>(p);
-    count_launch();
-    return cudaGetLastError();
+    return launch_pdl(prefill_sort_kernel, 1, 1024, 0, s, p);
 }
 
 cudaError_t launch_prefill_scatter(const PrefillScatterParams& p, cudaStream_t s) {
     const int nblk = (int)((p.T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
-    prefill_scatter_kernel<<<nblk, kRouteThreads, 0, s>>>(p);
-    count_launch();
-    return cudaGetLastError();
+    return launch_pdl(prefill_scatter_kernel, nblk, kRouteThreads, 0, s, p);
 }
 
 }  // namespace exfold
