@@ -312,15 +312,11 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     { ProfScope ps(0, s); EXFOLD_CUDA(launch_prefill_route(rp, s)); }
 
     const int nblk = (int)((T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
-    PrefillSortParams sp{};
-    sp.T = T; sp.N = N; sp.n_shared = l.n_shared; sp.Kp = Kp; sp.nblk = nblk;
-    sp.block_hist = rp.block_hist; sp.offsets = at<int32_t>(ws, pl.offsets);
-    sp.work_start = at<int32_t>(ws, pl.work_start); sp.totals = at<int32_t>(ws, pl.totals);
-    { ProfScope ps(1, s); EXFOLD_CUDA(launch_prefill_sort(sp, s)); }
-
     PrefillScatterParams cp{};
     cp.T = T; cp.N = N; cp.n_shared = l.n_shared; cp.Kp = Kp; cp.d_bytes = bf16 ? d * 2 : 0;
-    cp.ids = rp.ids; cp.w = rp.w; cp.block_hist = rp.block_hist; cp.offsets = sp.offsets;
+    cp.nblk = (int)((T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
+    cp.ids = rp.ids; cp.w = rp.w; cp.block_hist = rp.block_hist;
+    cp.offsets = at<int32_t>(ws, pl.offsets); cp.work_start = at<int32_t>(ws, pl.work_start);
     cp.x = x; cp.xs = bf16 ? at<char>(ws, pl.xs) : nullptr;
     cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
     cp.row_w = at<float>(ws, pl.row_w); cp.row_exp = at<int32_t>(ws, pl.row_exp);
@@ -330,7 +326,7 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     if (bf16) {
         GroupedGemmParams g{};
         g.tm_a = tm_xs; g.tm_a2 = tm_x; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu;
-        g.offsets = sp.offsets; g.work_start = sp.work_start; g.G = G; g.n_routed = N; g.R = (int)R;
+        g.offsets = cp.offsets; g.work_start = cp.work_start; g.G = G; g.n_routed = N; g.R = (int)R;
         g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.grp_expert = nullptr; g.n_groups_dev = nullptr;
         g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = cp.row_tok; g.row_w = cp.row_w;
         g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
@@ -356,7 +352,7 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
         if ((rc = copy_meta(meta->omit_src, rp.omit_src, (size_t)T * (K - Kp) * 4, s))) return rc;
         if ((rc = copy_meta(meta->omit_tgt, rp.omit_tgt, (size_t)T * (K - Kp) * 4, s))) return rc;
         if ((rc = copy_meta(meta->perm, cp.perm, (size_t)R * 4, s))) return rc;
-        if ((rc = copy_meta(meta->offsets, sp.offsets, (size_t)(N + 1) * 4, s))) return rc;
+        if ((rc = copy_meta(meta->offsets, cp.offsets, (size_t)(N + 1) * 4, s))) return rc;
     }
     return EXFOLD_OK;
 }

@@ -48,6 +48,29 @@ __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol
 void set_pdl(bool on);
 bool pdl_enabled();
 
+// Order-preserving map float -> uint32 (larger float <=> larger key), so warp arg-max / arg-min can use
+// the hardware integer reductions (redux.sync) instead of shuffle trees.
+__device__ __forceinline__ uint32_t float_order_key(float f) {
+    const uint32_t b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float float_from_order_key(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+// Warp-wide (value desc, id asc) arg-max. Lanes without a candidate pass has = false. Returns the
+// winning id to every lane and its key through *key_out. At least one lane must have a candidate.
+__device__ __forceinline__ int warp_argmax(bool has, uint32_t key, int id, uint32_t* key_out) {
+    const uint32_t m = __reduce_max_sync(0xffffffffu, has ? key : 0u);
+    const int best = __reduce_min_sync(0xffffffffu, (has && key == m) ? id : 0x7fffffff);
+    *key_out = m;
+    return best;
+}
+// Warp-wide (value asc, id asc) arg-min over lanes with has = true.
+__device__ __forceinline__ int warp_argmin(bool has, uint32_t key, int id) {
+    const uint32_t m = __reduce_min_sync(0xffffffffu, has ? key : 0xffffffffu);
+    return __reduce_min_sync(0xffffffffu, (has && key == m) ? id : 0x7fffffff);
+}
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
     cudaLaunchConfig_t cfg = {};
@@ -85,22 +108,15 @@ struct PrefillRouteParams {
 constexpr int kRouteTokensPerBlock = 64;
 constexpr int kRouteThreads = 512;
 
-struct PrefillSortParams {
-    int64_t T;
-    int N, n_shared, Kp, nblk;
-    int32_t* block_hist;  // [nblk][N] in: counts, out: exclusive prefix over blocks
-    int32_t* offsets;     // [G+1] sorted-row offsets (G = N + n_shared)
-    int32_t* work_start;  // [G+1] prefix of row tiles per group
-    int32_t* totals;      // [4]: total row tiles, total rows
-};
-
 struct PrefillScatterParams {
     int64_t T;
     int N, n_shared, Kp, d_bytes;  // d_bytes: bytes of one x row (0: no gather)
+    int nblk;                   // blocks of the route kernel (= blocks of this kernel)
     const int32_t* ids;         // [T][Kp]
     const float* w;             // [T][Kp]
-    const int32_t* block_hist;  // prefix form
-    const int32_t* offsets;
+    const int32_t* block_hist;  // [nblk][N] retained routes per (block, expert)
+    int32_t* offsets;           // [G+1] out: first sorted row of each group
+    int32_t* work_start;        // [G+1] out: prefix of 128-row tiles per group
     const void* x;      // [T][d]
     void* xs;           // [R][d] gathered rows (may be null)
     int32_t* perm;      // [R]
@@ -112,7 +128,6 @@ struct PrefillScatterParams {
 };
 
 cudaError_t launch_prefill_route(const PrefillRouteParams& p, cudaStream_t s);
-cudaError_t launch_prefill_sort(const PrefillSortParams& p, cudaStream_t s);
 cudaError_t launch_prefill_scatter(const PrefillScatterParams& p, cudaStream_t s);
 
 // ---------------------------------------------------------------- routing (decode)

@@ -41,40 +41,33 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     // ---- Eq. 2 per token (warp per token), weights in double
     for (int i = warp; i < B; i += kWarps) {
         const float* r = p.logits + (size_t)i * N;
-        float v[NPL];
+        uint32_t key_q[NPL];
         uint32_t used = 0;
 #pragma unroll
         for (int q = 0; q < NPL; ++q) {
-            int e = lane + 32 * q;
-            v[q] = e < N ? r[e] : -INFINITY;
+            const int e = lane + 32 * q;
+            key_q[q] = float_order_key(e < N ? r[e] : -INFINITY);
             if (e >= N) used |= 1u << q;
         }
         int my_id = -1;
         float my_r = 0.f;
         for (int k = 0; k < K; ++k) {
-            float bv = -INFINITY;
+            uint32_t bk = 0;
             int be = 0x7fffffff;
 #pragma unroll
             for (int q = 0; q < NPL; ++q) {
-                bool free_q = !((used >> q) & 1u);
-                if (free_q && (be == 0x7fffffff || v[q] > bv)) {
-                    bv = v[q];
+                const bool free_q = !((used >> q) & 1u);
+                if (free_q && (be == 0x7fffffff || key_q[q] > bk)) {
+                    bk = key_q[q];
                     be = lane + 32 * q;
                 }
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-                int oe = __shfl_xor_sync(0xffffffffu, be, off);
-                if (oe != 0x7fffffff && (be == 0x7fffffff || ov > bv || (ov == bv && oe < be))) {
-                    bv = ov;
-                    be = oe;
-                }
-            }
+            uint32_t mk;
+            be = warp_argmax(be != 0x7fffffff, bk, be, &mk);
             if ((be & 31) == lane) used |= 1u << (be >> 5);
             if (lane == k) {
                 my_id = be;
-                my_r = bv;
+                my_r = float_from_order_key(mk);
             }
         }
         const float rmax = __shfl_sync(0xffffffffu, my_r, 0);
@@ -149,15 +142,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
                 bt = t;
             }
         }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            float ol = __shfl_xor_sync(0xffffffffu, bl, off);
-            int ot = __shfl_xor_sync(0xffffffffu, bt, off);
-            if (ot != 0x7fffffff && (bt == 0x7fffffff || ol < bl || (ol == bl && ot < bt))) {
-                bl = ol;
-                bt = ot;
-            }
-        }
+        bt = warp_argmin(bt != 0x7fffffff, float_order_key(bl), bt);
         if (lane == 0) {
             sm.target[s] = bt;
             sm.scale[s] = __ldg(p.S + (size_t)s * N + bt);

@@ -4,11 +4,12 @@
 //   route kernel   one warp per token; lane l holds logits l, l+32, ...; after the Top-K
 //                  rounds lane k (k < K) owns route k. Writes ids/w/omitted pairs and a
 //                  per-block histogram of retained experts.
-//   sort kernel    one CTA: prefix over blocks per expert, prefix over experts -> offsets,
-//                  row-tile prefix for the GEMM work list.
-//   scatter kernel same token->block map as the route kernel; ranks routes inside the block in
-//                  (token, slot) order, so the permutation is the stable sort by expert and is
-//                  bit-reproducible; also gathers the token rows into sorted order.
+//   scatter kernel same token->block map as the route kernel. Each block first turns the block
+//                  histograms into its own bases (prefix over experts + prefix over earlier
+//                  blocks; block 0 also publishes offsets and the row-tile prefix for the GEMM
+//                  work list), then ranks its routes in (token, slot) order, so the permutation
+//                  is the stable sort by expert and is bit-reproducible; it also gathers the
+//                  token rows into sorted order and clears the fp32 accumulator.
 #include "common.cuh"
 
 namespace exfold {
@@ -29,45 +30,55 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_route_kernel(PrefillRou
 
     const int N = p.N, K = p.K, Kp = p.Kp, Ko = p.K - p.Kp;
     const int64_t tok0 = (int64_t)blockIdx.x * kRouteTokensPerBlock;
+    // the next token's logits are fetched while the current token is processed
+    float vn[NPL];
+    {
+        const int64_t i0 = tok0 + warp;
+#pragma unroll
+        for (int q = 0; q < NPL; ++q) {
+            const int e = lane + 32 * q;
+            vn[q] = (i0 < p.T && warp < kRouteTokensPerBlock && e < N) ? p.logits[i0 * N + e] : -INFINITY;
+        }
+    }
     for (int tl = warp; tl < kRouteTokensPerBlock; tl += kWarps) {
         const int64_t i = tok0 + tl;
         if (i >= p.T) break;
-        const float* r = p.logits + i * N;
-        float v[NPL];
+        uint32_t key_q[NPL];
         uint32_t used = 0;
 #pragma unroll
         for (int q = 0; q < NPL; ++q) {
-            int e = lane + 32 * q;
-            v[q] = e < N ? r[e] : -INFINITY;
-            if (e >= N) used |= 1u << q;
+            key_q[q] = float_order_key(vn[q]);
+            if (lane + 32 * q >= N) used |= 1u << q;
         }
-        // ---- Eq. 2: K rounds of warp arg-max; ties -> lower expert id
+        {
+            const int64_t in = i + kWarps;
+            const bool more = tl + kWarps < kRouteTokensPerBlock && in < p.T;
+#pragma unroll
+            for (int q = 0; q < NPL; ++q) {
+                const int e = lane + 32 * q;
+                vn[q] = (more && e < N) ? p.logits[in * N + e] : -INFINITY;
+            }
+        }
+        // ---- Eq. 2: K rounds of warp arg-max (hardware reductions); ties -> lower expert id
         int my_id = -1;
         float my_r = 0.f;
         for (int k = 0; k < K; ++k) {
-            float bv = -INFINITY;
+            uint32_t bk = 0;
             int be = 0x7fffffff;
 #pragma unroll
             for (int q = 0; q < NPL; ++q) {
-                bool free_q = !((used >> q) & 1u);
-                if (free_q && (be == 0x7fffffff || v[q] > bv)) {
-                    bv = v[q];
+                const bool free_q = !((used >> q) & 1u);
+                if (free_q && (be == 0x7fffffff || key_q[q] > bk)) {
+                    bk = key_q[q];
                     be = lane + 32 * q;
                 }
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-                int oe = __shfl_xor_sync(0xffffffffu, be, off);
-                if (oe != 0x7fffffff && (be == 0x7fffffff || ov > bv || (ov == bv && oe < be))) {
-                    bv = ov;
-                    be = oe;
-                }
-            }
+            uint32_t mk;
+            be = warp_argmax(be != 0x7fffffff, bk, be, &mk);
             if ((be & 31) == lane) used |= 1u << (be >> 5);
             if (lane == k) {
                 my_id = be;
-                my_r = bv;
+                my_r = float_from_order_key(mk);
             }
         }
         const bool has = lane < K;
@@ -89,30 +100,34 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_route_kernel(PrefillRou
         if (!has) rank = 0x7fff;
         const bool kept = has && rank < Kp;
         const bool omitted = has && rank >= Kp;
-        // ---- Eq. 12: each omitted route picks the retained expert with the smallest loss
-        float bl = INFINITY;
-        int bt = 0x7fffffff;
-        for (int j = 0; j < K; ++j) {
-            int ij = __shfl_sync(0xffffffffu, my_id, j);
-            int rj = __shfl_sync(0xffffffffu, rank, j);
-            if (omitted && rj < Kp) {
-                float l = __ldg(p.L + (size_t)my_id * N + ij);
-                if (bt == 0x7fffffff || l < bl || (l == bl && ij < bt)) {
-                    bl = l;
-                    bt = ij;
-                }
+        // ---- Eq. 12 + 13, omitted routes in rank order, four at a time. For an omitted source s every
+        // retained lane t loads L[s][t] and S[s][t] itself (independent loads, all in flight together);
+        // a warp arg-min over (loss, id) picks the target, which then adds w_s * S[s][t] to its weight.
+        float wt = w;
+        int my_tgt = -1;  // for omitted lanes: the chosen target
+        for (int rr0 = Kp; rr0 < K; rr0 += 4) {
+            int src_lane[4], src_id[4];
+            float lv[4], sv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int rr = rr0 + u;
+                const unsigned m = __ballot_sync(0xffffffffu, rank == rr);
+                src_lane[u] = m ? __ffs(m) - 1 : 0;
+                src_id[u] = __shfl_sync(0xffffffffu, my_id, src_lane[u]);
+                const bool act = kept && rr < K;
+                lv[u] = act ? __ldg(p.L + (size_t)src_id[u] * N + my_id) : INFINITY;
+                sv[u] = act ? __ldg(p.S + (size_t)src_id[u] * N + my_id) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (rr0 + u >= K) break;  // warp-uniform
+                const int bt = warp_argmin(kept, float_order_key(lv[u]), my_id);
+                const float ws = __shfl_sync(0xffffffffu, w, src_lane[u]);
+                if (kept && my_id == bt) wt = __fadd_rn(wt, __fmul_rn(ws, sv[u]));
+                if (lane == src_lane[u]) my_tgt = bt;
             }
         }
-        const float contrib = omitted ? __fmul_rn(w, __ldg(p.S + (size_t)my_id * N + bt)) : 0.f;
-        // ---- Eq. 13: add the omitted routes' scaled weights to their targets, in rank order
-        float wt = w;
-        for (int rr = Kp; rr < K; ++rr) {
-            unsigned m = __ballot_sync(0xffffffffu, rank == rr);
-            int src = __ffs(m) - 1;
-            float c = __shfl_sync(0xffffffffu, contrib, src);
-            int t = __shfl_sync(0xffffffffu, bt, src);
-            if (kept && my_id == t) wt = __fadd_rn(wt, c);
-        }
+        const int bt = my_tgt;
         if (kept) {
             p.ids[i * Kp + rank] = my_id;
             p.w[i * Kp + rank] = wt;
@@ -126,50 +141,12 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_route_kernel(PrefillRou
     for (int e = threadIdx.x; e < N; e += blockDim.x) p.block_hist[(size_t)blockIdx.x * N + e] = hist[e];
 }
 
-// One CTA. block_hist[b][e] (counts) -> exclusive prefix over blocks; offsets, work_start, totals.
-__global__ void __launch_bounds__(1024) prefill_sort_kernel(PrefillSortParams p) {
-    __shared__ int tot[kMaxGroups + 1];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const int N = p.N;
-    grid_dep_launch();
-    grid_dep_wait();
-    for (int e = warp; e < N; e += nwarps) {
-        int run = 0;
-        for (int b0 = 0; b0 < p.nblk; b0 += 32) {
-            int b = b0 + lane;
-            int c = b < p.nblk ? p.block_hist[(size_t)b * N + e] : 0;
-            int inc = c;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                int o = __shfl_up_sync(0xffffffffu, inc, off);
-                if (lane >= off) inc += o;
-            }
-            if (b < p.nblk) p.block_hist[(size_t)b * N + e] = run + inc - c;
-            run += __shfl_sync(0xffffffffu, inc, 31);
-        }
-        if (lane == 0) tot[e] = run;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int G = N + p.n_shared;
-        int off = 0, tiles = 0;
-        for (int g = 0; g < G; ++g) {
-            int rows = g < N ? tot[g] : (int)p.T;
-            p.offsets[g] = off;
-            p.work_start[g] = tiles;
-            off += rows;
-            tiles += (rows + kTileM - 1) / kTileM;
-        }
-        p.offsets[G] = off;
-        p.work_start[G] = tiles;
-        p.totals[0] = tiles;
-        p.totals[1] = off;
-    }
-}
-
 __global__ void __launch_bounds__(kRouteThreads) prefill_scatter_kernel(PrefillScatterParams p) {
     __shared__ int cnt[kMaxExperts];
     __shared__ int pos[kRouteTokensPerBlock * kMaxTopK];
+    __shared__ int part_pre[4][kMaxExperts];  // partial sums over blocks: before this block ...
+    __shared__ int part_tot[4][kMaxExperts];  // ... and over all blocks
+    __shared__ int tot[kMaxExperts];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int N = p.N, Kp = p.Kp;
     const int64_t tok0 = (int64_t)blockIdx.x * kRouteTokensPerBlock;
@@ -183,8 +160,41 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_scatter_kernel(PrefillS
         const int n4 = ntok * p.d / 4;
         for (int c = threadIdx.x; c < n4; c += blockDim.x) z[c] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    for (int e = threadIdx.x; e < N; e += blockDim.x)
-        cnt[e] = p.offsets[e] + p.block_hist[(size_t)blockIdx.x * N + e];
+    // Every block derives its own bases from the per-block histograms (a few KB, L2-resident): the
+    // first sorted position of expert e for this block is (rows of experts < e) + (rows of e in
+    // earlier blocks). No single-CTA scan kernel sits between routing and the GEMMs.
+    for (int idx = threadIdx.x; idx < 4 * N; idx += blockDim.x) {
+        const int e = idx % N, part = idx / N;
+        int pre = 0, all = 0;
+        for (int b = part; b < p.nblk; b += 4) {
+            const int h = p.block_hist[(size_t)b * N + e];
+            all += h;
+            if (b < (int)blockIdx.x) pre += h;
+        }
+        part_pre[part][e] = pre;
+        part_tot[part][e] = all;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < N; e += blockDim.x) tot[e] = part_tot[0][e] + part_tot[1][e] + part_tot[2][e] + part_tot[3][e];
+    __syncthreads();
+    for (int e = threadIdx.x; e < N; e += blockDim.x) {
+        int off = 0;
+        for (int o = 0; o < e; ++o) off += tot[o];
+        cnt[e] = off + part_pre[0][e] + part_pre[1][e] + part_pre[2][e] + part_pre[3][e];
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {  // group offsets and the row-tile prefix for the GEMM work list
+        const int G = N + p.n_shared;
+        int off = 0, tiles = 0;
+        for (int g = 0; g < G; ++g) {
+            const int rows = g < N ? tot[g] : (int)p.T;
+            p.offsets[g] = off;
+            p.work_start[g] = tiles;
+            off += rows;
+            tiles += (rows + kTileM - 1) / kTileM;
+        }
+        p.offsets[G] = off;
+        p.work_start[G] = tiles;
+    }
     __syncthreads();
     if (warp == 0) {
         // routes of this block in (token, slot) order, 32 at a time
@@ -243,10 +253,6 @@ cudaError_t launch_prefill_route(const PrefillRouteParams& p, cudaStream_t s) {
         case 3: case 4: return launch_pdl(prefill_route_kernel<4>, nblk, kRouteThreads, 0, s, p);
         default: return launch_pdl(prefill_route_kernel<8>, nblk, kRouteThreads, 0, s, p);
     }
-}
-
-cudaError_t launch_prefill_sort(const PrefillSortParams& p, cudaStream_t s) {
-    return launch_pdl(prefill_sort_kernel, 1, 1024, 0, s, p);
 }
 
 cudaError_t launch_prefill_scatter(const PrefillScatterParams& p, cudaStream_t s) {
