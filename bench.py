@@ -36,9 +36,9 @@ import synth_inputs as si  # noqa: E402
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes measured by ncu (dram__bytes_read.sum + dram__bytes_write.sum) divided by the algorithmic
 # bytes of the same launch, from the reduced-case captures summarised under profiles/
-# (gemm_prefill_mixtral_reduced.md, decode_ffn_mixtral_reduced.md). Traffic grows with the weights, so the
-# full-size figure is this ratio times the full-size algorithmic bytes.
-NCU_TRAFFIC_RATIO = {"gemm1": 511.8 / 502.3, "decode_gateup": 240.4 / 234.9}
+# (grouped_gemm_mixtral_reduced.md). Traffic grows with the weights, so the full-size figure is this ratio
+# times the full-size algorithmic bytes.
+NCU_TRAFFIC_RATIO = {"gemm1": 511.3 / 502.3, "decode_gateup": 239.3 / 234.9}
 
 
 def log(*a):
@@ -343,7 +343,7 @@ def run_ours(args, rank, world):
     if "decode_gateup" in kern:
         tg = kern["decode_gateup"] * 1e-3
         td = kern.get("decode_down", 0.0) * 1e-3
-        out["decode"]["roofline"] = {"kernel": "decode gate/up weight stream, tcgen05 swap-AB", "bound": "hbm",
+        out["decode"]["roofline"] = {"kernel": "decode GEMM-1 (gate/up weight stream over the pool), tcgen05", "bound": "hbm",
                                      "achieved": gateup_bytes / tg / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                      "frac": gateup_bytes / tg / 1e9 / peaks["hbm_gbs"],
                                      "traffic": gateup_bytes * NCU_TRAFFIC_RATIO["decode_gateup"],

@@ -4,10 +4,17 @@
 // by pool rank, duplicate (token, expert) slots merged ("routes folded into the same target
 // are coalesced before expert computation").
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace exfold {
 
 namespace {
+
+#ifdef EXFOLD_TRACE
+#define DEC_T(slot) if (threadIdx.x == 0) g_trace[2][0][slot] = ptx::globaltimer_ns()
+#else
+#define DEC_T(slot) ((void)0)
+#endif
 
 constexpr int kDecThreads = 1024;
 constexpr int kDecMaxSlots = 4096;
@@ -17,6 +24,7 @@ struct DecSmem {
     int ids[kDecMaxSlots];
     float wrm[kDecMaxSlots];  // remapped weights
     double score[kMaxExperts];
+    unsigned long long acc[kMaxExperts];  // sum_i w_{i,e} in fixed point (2^-53 units): exact, order-independent
     int in_union[kMaxExperts];
     int rank_of[kMaxExperts];   // pool rank or -1
     int pool[kMaxExperts];      // pool ids by rank
@@ -34,20 +42,46 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kDecThreads / 32;
     const int B = p.B, N = p.N, K = p.K, M = p.M;
+    DEC_T(0);
     grid_dep_launch();
     grid_dep_wait();
+    DEC_T(1);
     if (p.status != nullptr && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
+    // pull the loss and scalar tables towards L2 now; they are needed after the pool is known
+    {
+        const size_t table_bytes = (size_t)N * N * sizeof(float);
+        for (size_t off = (size_t)threadIdx.x * 128; off < table_bytes; off += (size_t)kDecThreads * 128) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(p.L) + off));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(p.S) + off));
+        }
+    }
 
-    // ---- Eq. 2 per token (warp per token), weights in double
+    for (int e = threadIdx.x; e < N; e += kDecThreads) {
+        sm.acc[e] = 0ull;
+        sm.in_union[e] = 0;
+    }
+    __syncthreads();
+    // ---- Eq. 2 per token (warp per token), weights in double; the next token's logits are fetched
+    // while the current one is processed. Each route adds its weight to its expert's fixed-point
+    // accumulator (integer atomics: the sum does not depend on the order of arrival).
+    float vn[NPL];
+#pragma unroll
+    for (int q = 0; q < NPL; ++q) {
+        const int e = lane + 32 * q;
+        vn[q] = (warp < B && e < N) ? p.logits[(size_t)warp * N + e] : -INFINITY;
+    }
     for (int i = warp; i < B; i += kWarps) {
-        const float* r = p.logits + (size_t)i * N;
         uint32_t key_q[NPL];
         uint32_t used = 0;
 #pragma unroll
         for (int q = 0; q < NPL; ++q) {
+            key_q[q] = float_order_key(vn[q]);
+            if (lane + 32 * q >= N) used |= 1u << q;
+        }
+#pragma unroll
+        for (int q = 0; q < NPL; ++q) {
             const int e = lane + 32 * q;
-            key_q[q] = float_order_key(e < N ? r[e] : -INFINITY);
-            if (e >= N) used |= 1u << q;
+            vn[q] = (i + kWarps < B && e < N) ? p.logits[(size_t)(i + kWarps) * N + e] : -INFINITY;
         }
         int my_id = -1;
         float my_r = 0.f;
@@ -75,80 +109,94 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         double sum = 0.0;
         for (int k = 0; k < K; ++k) sum += __shfl_sync(0xffffffffu, ex, k);  // slot order, like the definition
         if (lane < K) {
+            const double wv = ex / sum;
             sm.ids[i * K + lane] = my_id;
-            sm.w64[i * K + lane] = ex / sum;
+            sm.w64[i * K + lane] = wv;
+            atomicAdd(&sm.acc[my_id], (unsigned long long)(wv * 9007199254740992.0));  // 2^53
+            sm.in_union[my_id] = 1;
         }
     }
     __syncthreads();
+    DEC_T(2);
 
-    // ---- Eq. 11: union and score_e = h_e * sum_i w_{i,e} (double; fixed reduction order)
+    // ---- Eq. 11: score_e = h_e * sum_i w_{i,e}
     const int nslots = B * K;
-    for (int e = warp; e < N; e += kWarps) {
-        double acc = 0.0;
-        int cnt = 0;
-        for (int s = lane; s < nslots; s += 32)
-            if (sm.ids[s] == e) {
-                acc += sm.w64[s];
-                cnt++;
-            }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
-        }
-        if (lane == 0) {
-            sm.score[e] = acc * (double)p.h[e];
-            sm.in_union[e] = cnt > 0;
-        }
-    }
+    for (int e = threadIdx.x; e < N; e += kDecThreads)
+        sm.score[e] = (double)sm.acc[e] * (1.0 / 9007199254740992.0) * (double)p.h[e];
     __syncthreads();
-    // pool = best min(M, |U|) experts of the union by (score desc, id asc)
+    DEC_T(3);
+    // pool = best min(M, |U|) experts of the union by (score desc, id asc): rank by counting,
+    // four threads per expert
     {
-        int e = threadIdx.x;
-        int in_u = (e < N) ? sm.in_union[e] : 0;
-        int usize = __syncthreads_count(in_u);
-        if (e < N) {
-            int rk = -1;
-            if (in_u) {
-                rk = 0;
-                const double se = sm.score[e];
-                for (int o = 0; o < N; ++o)
-                    if (sm.in_union[o] && (sm.score[o] > se || (sm.score[o] == se && o < e))) rk++;
-                if (rk >= M) rk = -1;
-            }
+        const int e = threadIdx.x >> 2, part = threadIdx.x & 3;  // 1024 threads cover 256 experts
+        const int in_u = (e < N) ? sm.in_union[e] : 0;
+        int better = 0;
+        if (in_u) {
+            const double se = sm.score[e];
+            for (int o = part; o < N; o += 4)
+                if (sm.in_union[o] && (sm.score[o] > se || (sm.score[o] == se && o < e))) better++;
+        }
+        better += __shfl_xor_sync(0xffffffffu, better, 1);
+        better += __shfl_xor_sync(0xffffffffu, better, 2);
+        const int usize = __syncthreads_count(in_u && part == 0);
+        if (e < N && part == 0) {
+            const int rk = (in_u && better < M) ? better : -1;
             sm.rank_of[e] = rk;
             if (rk >= 0) sm.pool[rk] = e;
         }
         if (threadIdx.x == 0) sm.P = usize < M ? usize : M;
     }
     __syncthreads();
+    DEC_T(4);
     const int P = sm.P;
-    // ---- Eq. 12 for every source expert: itself if in the pool, else its min-loss pool expert
-    for (int s = warp; s < N; s += kWarps) {
-        if (sm.rank_of[s] >= 0) {
-            if (lane == 0) {
-                sm.target[s] = s;
-                sm.scale[s] = 1.0f;
+    // ---- Eq. 12 for every source expert: itself if in the pool, else its min-loss pool expert.
+    // A warp takes up to 8 sources at a time and issues all their loss loads before reducing, then
+    // all their scalar loads: two rounds of memory latency per batch instead of two per source.
+    for (int s0 = warp * 8; s0 < N; s0 += kWarps * 8) {
+        float bl[8];
+        int bt[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int s = s0 + u;
+            bl[u] = INFINITY;
+            bt[u] = 0x7fffffff;
+            if (s < N && sm.rank_of[s] < 0) {
+                for (int j = lane; j < P; j += 32) {
+                    const int t = sm.pool[j];
+                    const float l = __ldg(p.L + (size_t)s * N + t);
+                    if (bt[u] == 0x7fffffff || l < bl[u] || (l == bl[u] && t < bt[u])) {
+                        bl[u] = l;
+                        bt[u] = t;
+                    }
+                }
             }
-            continue;
         }
-        float bl = INFINITY;
-        int bt = 0x7fffffff;
-        for (int j = lane; j < P; j += 32) {
-            int t = sm.pool[j];
-            float l = __ldg(p.L + (size_t)s * N + t);
-            if (bt == 0x7fffffff || l < bl || (l == bl && t < bt)) {
-                bl = l;
-                bt = t;
+        float sc[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int s = s0 + u;
+            sc[u] = 1.0f;
+            if (s < N) {  // warp-uniform
+                if (sm.rank_of[s] >= 0) bt[u] = s;
+                else {
+                    bt[u] = warp_argmin(bt[u] != 0x7fffffff, float_order_key(bl[u]), bt[u]);
+                    if (lane == 0) sc[u] = __ldg(p.S + (size_t)s * N + bt[u]);
+                }
             }
         }
-        bt = warp_argmin(bt != 0x7fffffff, float_order_key(bl), bt);
         if (lane == 0) {
-            sm.target[s] = bt;
-            sm.scale[s] = __ldg(p.S + (size_t)s * N + bt);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int s = s0 + u;
+                if (s < N) {
+                    sm.target[s] = bt[u];
+                    sm.scale[s] = sc[u];
+                }
+            }
         }
     }
     __syncthreads();
+    DEC_T(5);
     // ---- Eq. 14: remap every slot in place; [B][K] layout kept
     for (int s = threadIdx.x; s < nslots; s += kDecThreads) {
         int e = sm.ids[s];
@@ -174,6 +222,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     }
     if (threadIdx.x == 0) *p.pool_size = P;
     __syncthreads();
+    DEC_T(6);
     // ---- execution lists: one row per distinct (token, pool expert), grouped by pool rank
     for (int pass = 0; pass < 2; ++pass) {
         for (int g = warp; g < P; g += kWarps) {
@@ -213,6 +262,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
             __syncthreads();
         }
     }
+    DEC_T(7);
     const int G = P + (p.n_shared ? 1 : 0);
     for (int g = threadIdx.x; g <= G; g += kDecThreads) {
         p.grp_off[g] = sm.goff[g];
@@ -235,6 +285,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         p.n_groups[0] = G;
         p.n_groups[1] = sm.goff[G];  // total rows
     }
+    DEC_T(8);
 }
 
 // xs[row] = x[row_tok[row]] for row < n_rows (device value); CTAs with blockIdx < zero_rows also
