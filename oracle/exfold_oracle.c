@@ -500,6 +500,60 @@ int orc_decode_fold(const float *logits, int64_t B, int N, int K, int M, const f
 }
 
 /*
+ * Static decode pool (appendix, "static implementation"): the pool is formed once from the
+ * calibration-time norms, pool = TopK_e(h_e, M) over ALL experts (ties -> lower id, listed in
+ * descending h), and one target and one scalar are precomputed for every possible source expert:
+ * target[s] = s, scale[s] = 1 inside the pool, else the minimum-loss pool expert and S[s][target].
+ */
+int orc_static_pool(int N, int M, const float *S, const float *L, const float *h, int32_t *pool_ids,
+                    int32_t *target, float *scale)
+{
+    if (M < 1 || M > N) return -1;
+    char *in_pool = (char *)calloc((size_t)N, 1);
+    if (!in_pool) return -3;
+    for (int j = 0; j < M; ++j) {
+        int best = -1;
+        for (int e = 0; e < N; ++e) {
+            if (in_pool[e]) continue;
+            if (best < 0 || h[e] > h[best]) best = e; /* strict >: lower id wins ties */
+        }
+        pool_ids[j] = best;
+        in_pool[best] = 1;
+    }
+    for (int s = 0; s < N; ++s) {
+        if (in_pool[s]) { target[s] = s; scale[s] = 1.0f; }
+        else {
+            int t = argmin_loss(L, N, s, pool_ids, M);
+            target[s] = t;
+            scale[s] = S[(size_t)s * N + t];
+        }
+    }
+    free(in_pool);
+    return 0;
+}
+
+/*
+ * Per-route remapping with precomputed tables (the appendix's remapping listing): every routed
+ * slot (id, w) of Eq. 2 becomes (target[id], w * scale[id]); the [B][K] layout is kept.
+ */
+int orc_decode_static(const float *logits, int64_t B, int N, int K, const int32_t *target,
+                      const float *scale, int32_t *ids_out, float *w_out)
+{
+    if (K < 1 || K > 64 || K > N) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < B; ++i) {
+        int32_t ids[64];
+        double w[64];
+        gate_token(logits + i * N, N, K, ids, w);
+        for (int k = 0; k < K; ++k) {
+            ids_out[i * K + k] = target[ids[k]];
+            w_out[i * K + k] = (float)(w[k] * (double)scale[ids[k]]);
+        }
+    }
+    return 0;
+}
+
+/*
  * Eq. 4 written out for decode, given the pool: retained routes run their own expert,
  * routes outside the pool run their minimum-loss pool expert scaled by S. Nothing merged.
  */

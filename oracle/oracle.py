@@ -203,3 +203,27 @@ def sort_routes(ids, n_groups: int):
     rc = _L().orc_sort_routes(_p(flat), C.c_int64(R), n_groups, _p(perm), _p(offsets))
     assert rc == 0, rc
     return perm, offsets
+
+
+def static_pool(M: int, S, L, h):
+    """Static decode pool from the calibration norms. Returns dict(pool_ids [M], target [N], scale [N])."""
+    S, L, h = _c(S, np.float32), _c(L, np.float32), _c(h, np.float32)
+    N = h.shape[0]
+    pool_ids = np.empty(M, np.int32)
+    target = np.empty(N, np.int32)
+    scale = np.empty(N, np.float32)
+    rc = _L().orc_static_pool(N, M, _p(S), _p(L), _p(h), _p(pool_ids), _p(target), _p(scale))
+    assert rc == 0, rc
+    return dict(pool_ids=pool_ids, target=target, scale=scale)
+
+
+def decode_static(logits, K: int, target, scale):
+    """Per-route remap with precomputed target/scale tables. Returns dict(ids [B,K], w [B,K])."""
+    logits = _c(logits, np.float32)
+    target, scale = _c(target, np.int32), _c(scale, np.float32)
+    B, N = logits.shape
+    ids = np.empty((B, K), np.int32)
+    w = np.empty((B, K), np.float32)
+    rc = _L().orc_decode_static(_p(logits), C.c_int64(B), N, K, _p(target), _p(scale), _p(ids), _p(w))
+    assert rc == 0, rc
+    return dict(ids=ids, w=w)

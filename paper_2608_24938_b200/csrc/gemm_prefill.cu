@@ -31,7 +31,7 @@ constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;
 
 struct WorkItem {
-    int g, row0, rows, n_idx, kpart;
+    int g, row0, rows, n_idx, kpart, m_idx;
 };
 
 // Work index -> (group, row tile, column tile, K part). Order: group, column tile, row tile, K part
@@ -52,6 +52,7 @@ __device__ __forceinline__ WorkItem decode_work(int w_all, int G, int nt, int ks
     const int tiles = s_ws[lo + 1] - s_ws[lo];
     const int local = w - s_ws[lo] * nt;
     const int m_idx = local % tiles;
+    it.m_idx = m_idx;
     it.n_idx = local / tiles;
     it.row0 = s_off[lo] + m_idx * kTileM;
     const int left = s_off[lo + 1] - it.row0;

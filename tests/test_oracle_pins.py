@@ -238,6 +238,38 @@ def test_decode_pool_invariants_and_listing_semantics():
                 assert scl[s] == S[s, tgt[s]]
 
 
+def test_static_pool_and_listing_remap():
+    """Static pool = the M experts with the largest calibration norm; per-route remap = the appendix
+    listing (two table lookups, one multiply per slot); with the dynamic pool's tables the static remap
+    reproduces the dynamic one; M = N is the unfolded layer."""
+    g = np.random.default_rng(16)
+    N, K, B = 16, 4, 20
+    lg = g.standard_normal((B, N)).astype(np.float32)
+    S, L, h, lnh = rand_tables(N, 8, unobs=0.05)
+    h[3] = h[9]  # a tie in the norms: the lower id must win
+    ids, w, w64 = oracle.gate(lg, K)
+    for M in (1, 5, 16):
+        sp = oracle.static_pool(M, S, L, h)
+        order = sorted(range(N), key=lambda e: (-float(h[e]), e))
+        assert sp["pool_ids"].tolist() == order[:M]
+        pool = sorted(order[:M])
+        for s in range(N):
+            if s in pool:
+                assert sp["target"][s] == s and sp["scale"][s] == 1
+            else:
+                assert sp["target"][s] == pool[int(np.argmin([L[s, c] for c in pool]))]
+                assert sp["scale"][s] == S[s, sp["target"][s]]
+        dec = oracle.decode_static(lg, K, sp["target"], sp["scale"])
+        assert np.array_equal(dec["ids"], sp["target"][ids])
+        assert np.array_equal(dec["w"], (w64 * sp["scale"][ids].astype(np.float64)).astype(np.float32))
+        assert np.isin(dec["ids"], pool).all()
+        if M == N:
+            assert np.array_equal(dec["ids"], ids) and np.array_equal(dec["w"], w)
+    dyn = oracle.decode_fold(lg, K, 5, S, L, h)
+    st = oracle.decode_static(lg, K, dyn["target"], dyn["scale"])
+    assert np.array_equal(st["ids"], dyn["ids"]) and np.array_equal(st["w"], dyn["w"])
+
+
 def test_single_token_decode_equals_prefill():
     """B = 1: Eq. 11 reduces to Eq. 10 with K' = M, so both modes give the same output."""
     cfg, x, lg, wg, wu, wd = tiny_layer(seed=15, N=8, T=6)
