@@ -153,6 +153,31 @@ int exfold_moe_decode(const exfold_layer *layer, const void *x, const float *log
                       const exfold_decode_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Static decode pool (appendix, "static implementation"): the pool is formed once from the
+ * calibration-time norms, pool = TopK_e(h_e, M) over all routed experts (ties -> lower id), and
+ * one target and one scalar are cached for every possible source expert, which removes the
+ * per-step batch reduction of Eq. 11. exfold_static_pool_build fills the caller's device arrays;
+ * exfold_moe_decode_static then runs a decode step whose routing is the per-route remap of the
+ * appendix listing (out_id = target[id], out_w = w * scale[id], [B][K] layout kept) followed by
+ * the expert FFN over the pool experts that received rows. Metadata, workspace, stream and
+ * error conventions are those of exfold_moe_decode; pool experts without a route this step are
+ * not read.
+ */
+typedef struct {
+    int32_t *pool_ids; /* [pool_m] pool experts, descending h           */
+    int32_t *target;   /* [N]  s itself if in the pool, else its minimum-loss pool expert */
+    float *scale;      /* [N]  1 or S[s][target[s]]                     */
+    int32_t pool_m;    /* M in [1, N]                                   */
+} exfold_static_pool;
+
+int exfold_static_pool_build(const exfold_layer *layer, const exfold_tables *tables, int32_t pool_m,
+                             exfold_static_pool *out, void *cuda_stream);
+int exfold_moe_decode_static(const exfold_layer *layer, const void *x, const float *logits, int64_t B,
+                             const void *w_gate, const void *w_up, const void *w_down,
+                             const exfold_static_pool *pool, void *y, const exfold_decode_meta *meta,
+                             void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * The same two calls for activations that live in HOST memory (pinned for real overlap):
  * x_host, logits_host and y_host are host pointers; the call stages them through the
  * workspace with asynchronous copies on the stream (x and logits in before the layer, y out

@@ -29,7 +29,7 @@ EXFOLD_WARN_UNOBSERVED_EXPERT = 1
 EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibrate", "exfold_moe_prefill",
            "exfold_moe_decode", "exfold_moe_prefill_host", "exfold_moe_decode_host", "exfold_device_status",
            "exfold_status_string", "exfold_launch_count", "exfold_profile_enable", "exfold_profile_read",
-           "exfold_moe_decode_noalloc"]
+           "exfold_moe_decode_noalloc", "exfold_static_pool_build", "exfold_moe_decode_static"]
 PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
                  "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
                  "simt_combine"]
@@ -59,6 +59,10 @@ class exfold_decode_meta(C.Structure):
                 ("w", C.c_void_p), ("target", C.c_void_p), ("scale", C.c_void_p)]
 
 
+class exfold_static_pool(C.Structure):
+    _fields_ = [("pool_ids", C.c_void_p), ("target", C.c_void_p), ("scale", C.c_void_p), ("pool_m", C.c_int32)]
+
+
 def _load() -> C.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2608_24938_b200.build` "
@@ -83,6 +87,12 @@ def _load() -> C.CDLL:
     lib.exfold_moe_decode_noalloc.restype = C.c_int
     lib.exfold_moe_decode_noalloc.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables),
                                               i32, vp, C.POINTER(exfold_decode_meta), vp]
+    lib.exfold_static_pool_build.restype = C.c_int
+    lib.exfold_static_pool_build.argtypes = [C.POINTER(exfold_layer), C.POINTER(exfold_tables), i32,
+                                             C.POINTER(exfold_static_pool), vp]
+    lib.exfold_moe_decode_static.restype = C.c_int
+    lib.exfold_moe_decode_static.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp,
+                                             C.POINTER(exfold_static_pool), vp, C.POINTER(exfold_decode_meta), vp, sz, vp]
     lib.exfold_device_status.restype = C.c_int
     lib.exfold_device_status.argtypes = [vp, vp]
     lib.exfold_status_string.restype = C.c_char_p
@@ -250,4 +260,25 @@ def exfold_moe_decode_noalloc(layer, x, logits, w_gate, w_up, w_down, tables: ex
                                        _stream(stream))
     if check and rc != 0:
         raise ExfoldError(rc, "exfold_moe_decode_noalloc")
+    return rc
+
+
+def exfold_static_pool_build(layer, tables: exfold_tables, pool_m: int, pool_ids, target, scale,
+                             stream=None) -> exfold_static_pool:
+    """Fills the caller's device arrays pool_ids [M], target [N], scale [N] and returns the struct to pass to
+    exfold_moe_decode_static (the tensors must stay alive as long as the struct is used)."""
+    sp = exfold_static_pool(_ptr(pool_ids), _ptr(target), _ptr(scale), pool_m)
+    rc = lib.exfold_static_pool_build(C.byref(layer), C.byref(tables), pool_m, C.byref(sp), _stream(stream))
+    if rc != 0:
+        raise ExfoldError(rc, "exfold_static_pool_build")
+    return sp
+
+
+def exfold_moe_decode_static(layer, x, logits, w_gate, w_up, w_down, pool: exfold_static_pool, y, ws,
+                             meta: Optional[dict] = None, stream=None, check: bool = True) -> int:
+    rc = lib.exfold_moe_decode_static(C.byref(layer), _ptr(x), _ptr(logits), x.shape[0], _ptr(w_gate), _ptr(w_up),
+                                      _ptr(w_down), C.byref(pool), _ptr(y), _decode_meta(meta), _ptr(ws), ws.numel(),
+                                      _stream(stream))
+    if check and rc != 0:
+        raise ExfoldError(rc, "exfold_moe_decode_static")
     return rc

@@ -357,9 +357,18 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     return EXFOLD_OK;
 }
 
-int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* logits, int64_t B, const void* w_gate,
-                      const void* w_up, const void* w_down, const exfold_tables* tables, int32_t pool_m, void* y,
-                      const exfold_decode_meta* meta, void* ws, size_t ws_bytes, void* cuda_stream) {
+// Dynamic (tables != null) or static (spool != null) decode step.
+static int decode_impl(const exfold_layer* layer, const void* x, const float* logits, int64_t B, const void* w_gate,
+                       const void* w_up, const void* w_down, const exfold_tables* tables,
+                       const exfold_static_pool* spool, int32_t pool_m, void* y, const exfold_decode_meta* meta,
+                       void* ws, size_t ws_bytes, void* cuda_stream) {
+    exfold_tables dummy{};  // the static path needs no tables: satisfy the common pointer checks
+    if (spool != nullptr) {
+        if (!spool->pool_ids || !spool->target || !spool->scale) return EXFOLD_ERR_INVALID_ARG;
+        dummy.S = dummy.L = dummy.h = dummy.lnh = spool->scale;
+        tables = &dummy;
+        pool_m = spool->pool_m;
+    }
     int rc = check_common(layer, x, logits, B, w_gate, w_up, w_down, tables, y, ws);
     if (rc != EXFOLD_OK) return rc;
     const exfold_layer& l = *layer;
@@ -390,6 +399,9 @@ int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* log
     DecodeRouteParams rp{};
     rp.logits = logits; rp.S = tables->S; rp.L = tables->L; rp.h = tables->h;
     rp.B = (int)B; rp.N = N; rp.K = K; rp.M = pool_m; rp.n_shared = l.n_shared;
+    if (spool != nullptr) {
+        rp.st_pool = spool->pool_ids; rp.st_target = spool->target; rp.st_scale = spool->scale;
+    }
     rp.pool_ids = at<int32_t>(ws, pl.pool_ids); rp.pool_size = at<int32_t>(ws, pl.pool_size);
     rp.pool_mask = at<uint32_t>(ws, pl.pool_mask); rp.ids = at<int32_t>(ws, pl.ids); rp.w = at<float>(ws, pl.w);
     rp.target = at<int32_t>(ws, pl.target); rp.scale = at<float>(ws, pl.scale);
@@ -444,6 +456,32 @@ int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* log
         if ((rc = copy_meta(meta->target, rp.target, (size_t)N * 4, s))) return rc;
         if ((rc = copy_meta(meta->scale, rp.scale, (size_t)N * 4, s))) return rc;
     }
+    return EXFOLD_OK;
+}
+
+int exfold_moe_decode(const exfold_layer* layer, const void* x, const float* logits, int64_t B, const void* w_gate,
+                      const void* w_up, const void* w_down, const exfold_tables* tables, int32_t pool_m, void* y,
+                      const exfold_decode_meta* meta, void* ws, size_t ws_bytes, void* cuda_stream) {
+    return decode_impl(layer, x, logits, B, w_gate, w_up, w_down, tables, nullptr, pool_m, y, meta, ws, ws_bytes,
+                       cuda_stream);
+}
+
+int exfold_moe_decode_static(const exfold_layer* layer, const void* x, const float* logits, int64_t B,
+                             const void* w_gate, const void* w_up, const void* w_down, const exfold_static_pool* pool,
+                             void* y, const exfold_decode_meta* meta, void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (pool == nullptr) return EXFOLD_ERR_INVALID_ARG;
+    return decode_impl(layer, x, logits, B, w_gate, w_up, w_down, nullptr, pool, pool->pool_m, y, meta, ws, ws_bytes,
+                       cuda_stream);
+}
+
+int exfold_static_pool_build(const exfold_layer* layer, const exfold_tables* tables, int32_t pool_m,
+                             exfold_static_pool* out, void* cuda_stream) {
+    if (!valid_layer(layer) || !tables || !tables->S || !tables->L || !tables->h || !out) return EXFOLD_ERR_INVALID_ARG;
+    if (!out->pool_ids || !out->target || !out->scale) return EXFOLD_ERR_INVALID_ARG;
+    if (pool_m < 1 || pool_m > layer->n_experts) return EXFOLD_ERR_INVALID_ARG;
+    out->pool_m = pool_m;
+    EXFOLD_CUDA(launch_static_pool(layer->n_experts, pool_m, tables->S, tables->L, tables->h, out->pool_ids,
+                                   out->target, out->scale, reinterpret_cast<cudaStream_t>(cuda_stream)));
     return EXFOLD_OK;
 }
 

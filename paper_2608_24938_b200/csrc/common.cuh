@@ -137,6 +137,10 @@ struct DecodeRouteParams {
     const float* L;
     const float* h;
     int B, N, K, M, n_shared;
+    // static pool (all null for the dynamic pool of Eq. 11): precomputed pool, targets and scalars
+    const int32_t* st_pool;    // [M]
+    const int32_t* st_target;  // [N]
+    const float* st_scale;     // [N]
     // metadata (workspace copies)
     int32_t* pool_ids;    // [N] (-1 padded)
     int32_t* pool_size;   // [1]
@@ -155,6 +159,8 @@ struct DecodeRouteParams {
     DeviceStatus* status; // cleared here (first kernel of a decode call)
 };
 cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s);
+cudaError_t launch_static_pool(int N, int M, const float* S, const float* L, const float* h, int32_t* pool_ids,
+                               int32_t* target, float* scale, cudaStream_t s);
 cudaError_t launch_gather_rows(const void* x, const int32_t* row_tok, const int32_t* n_rows_ptr, int max_rows,
                                int row_bytes, void* xs, float* y32, int zero_rows, int zero_row_floats,
                                cudaStream_t s);

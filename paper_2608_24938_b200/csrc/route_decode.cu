@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     DEC_T(1);
     if (p.status != nullptr && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
     // pull the loss and scalar tables towards L2 now; they are needed after the pool is known
-    {
+    if (p.st_pool == nullptr) {
         const size_t table_bytes = (size_t)N * N * sizeof(float);
         for (size_t off = (size_t)threadIdx.x * 128; off < table_bytes; off += (size_t)kDecThreads * 128) {
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(p.L) + off));
@@ -119,15 +119,32 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     __syncthreads();
     DEC_T(2);
 
-    // ---- Eq. 11: score_e = h_e * sum_i w_{i,e}
     const int nslots = B * K;
-    for (int e = threadIdx.x; e < N; e += kDecThreads)
-        sm.score[e] = (double)sm.acc[e] * (1.0 / 9007199254740992.0) * (double)p.h[e];
+    const bool is_static = p.st_pool != nullptr;
+    if (is_static) {
+        // static pool: precomputed pool, targets and scalars; no batch reduction
+        for (int e = threadIdx.x; e < N; e += kDecThreads) {
+            sm.rank_of[e] = -1;
+            sm.target[e] = p.st_target[e];
+            sm.scale[e] = p.st_scale[e];
+        }
+        __syncthreads();
+        for (int j = threadIdx.x; j < M; j += kDecThreads) {
+            const int e = p.st_pool[j];
+            sm.pool[j] = e;
+            sm.rank_of[e] = j;
+        }
+        if (threadIdx.x == 0) sm.P = M;
+    }
+    // ---- Eq. 11: score_e = h_e * sum_i w_{i,e}
+    if (!is_static)
+        for (int e = threadIdx.x; e < N; e += kDecThreads)
+            sm.score[e] = (double)sm.acc[e] * (1.0 / 9007199254740992.0) * (double)p.h[e];
     __syncthreads();
     DEC_T(3);
     // pool = best min(M, |U|) experts of the union by (score desc, id asc): rank by counting,
     // four threads per expert
-    {
+    if (!is_static) {
         const int e = threadIdx.x >> 2, part = threadIdx.x & 3;  // 1024 threads cover 256 experts
         const int in_u = (e < N) ? sm.in_union[e] : 0;
         int better = 0;
@@ -152,7 +169,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     // ---- Eq. 12 for every source expert: itself if in the pool, else its min-loss pool expert.
     // A warp takes up to 8 sources at a time and issues all their loss loads before reducing, then
     // all their scalar loads: two rounds of memory latency per batch instead of two per source.
-    for (int s0 = warp * 8; s0 < N; s0 += kWarps * 8) {
+    for (int s0 = warp * 8; s0 < N && !is_static; s0 += kWarps * 8) {
         float bl[8];
         int bt[8];
 #pragma unroll
@@ -288,6 +305,55 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     DEC_T(8);
 }
 
+// Static pool: pool = TopK_e(h_e, M) (ties -> lower id, descending h), then Eq. 12 for every source.
+__global__ void __launch_bounds__(256) static_pool_kernel(int N, int M, const float* __restrict__ S,
+                                                          const float* __restrict__ L, const float* __restrict__ h,
+                                                          int32_t* pool_ids, int32_t* target, float* scale) {
+    __shared__ int pool[kMaxExperts];
+    __shared__ int rank_of[kMaxExperts];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    grid_dep_launch();
+    grid_dep_wait();
+    for (int e = threadIdx.x; e < N; e += blockDim.x) {
+        const float he = h[e];
+        int better = 0;
+        for (int o = 0; o < N; ++o) {
+            const float ho = h[o];
+            if (ho > he || (ho == he && o < e)) better++;
+        }
+        rank_of[e] = better < M ? better : -1;
+        if (better < M) {
+            pool[better] = e;
+            pool_ids[better] = e;
+        }
+    }
+    __syncthreads();
+    for (int s = warp; s < N; s += nwarps) {
+        if (rank_of[s] >= 0) {
+            if (lane == 0) {
+                target[s] = s;
+                scale[s] = 1.0f;
+            }
+            continue;
+        }
+        float bl = INFINITY;
+        int bt = 0x7fffffff;
+        for (int j = lane; j < M; j += 32) {
+            const int t = pool[j];
+            const float l = L[(size_t)s * N + t];
+            if (bt == 0x7fffffff || l < bl || (l == bl && t < bt)) {
+                bl = l;
+                bt = t;
+            }
+        }
+        bt = warp_argmin(bt != 0x7fffffff, float_order_key(bl), bt);
+        if (lane == 0) {
+            target[s] = bt;
+            scale[s] = S[(size_t)s * N + bt];
+        }
+    }
+}
+
 // xs[row] = x[row_tok[row]] for row < n_rows (device value); CTAs with blockIdx < zero_rows also
 // clear one row of the fp32 accumulator y32.
 __global__ void __launch_bounds__(256) gather_rows_kernel(const void* __restrict__ x,
@@ -328,6 +394,11 @@ cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s) {
     }
 #undef EXFOLD_DEC_LAUNCH
     return err;
+}
+
+cudaError_t launch_static_pool(int N, int M, const float* S, const float* L, const float* h, int32_t* pool_ids,
+                               int32_t* target, float* scale, cudaStream_t s) {
+    return launch_pdl(static_pool_kernel, 1, 256, 0, s, N, M, S, L, h, pool_ids, target, scale);
 }
 
 cudaError_t launch_gather_rows(const void* x, const int32_t* row_tok, const int32_t* n_rows_ptr, int max_rows,

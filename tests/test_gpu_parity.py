@@ -170,6 +170,41 @@ def test_decode_max_batch_and_all_unobserved_row():
     check_output(got["y"], ref["y"], "bf16")
 
 
+@pytest.mark.parametrize("n_shared,M", [(0, 5), (1, 3), (0, 16)])
+def test_static_pool_decode(n_shared, M):
+    """Static pool built on the GPU equals the oracle's; a decode step with it equals the per-route
+    remap followed by the expert FFN."""
+    cfg = small_bf16(n_shared=n_shared, decode_batch=40)
+    case = Case(cfg)
+    ex, dev = case.ex, case.dev
+    N, K, B = cfg.n_experts, cfg.top_k, case.B
+    S, L, h, lnh = case.np_tables()
+    ref_pool = oracle.static_pool(M, S, L, h)
+    pool_ids = torch.full((M,), -7, dtype=torch.int32, device=dev)
+    target = torch.full((N,), -7, dtype=torch.int32, device=dev)
+    scale = torch.full((N,), float("nan"), dtype=torch.float32, device=dev)
+    sp = ex.exfold_static_pool_build(case.layer, case.tables, M, pool_ids, target, scale)
+    torch.cuda.synchronize()
+    assert np.array_equal(pool_ids.cpu().numpy(), ref_pool["pool_ids"])
+    assert np.array_equal(target.cpu().numpy(), ref_pool["target"])
+    assert np.array_equal(scale.cpu().numpy(), ref_pool["scale"])
+    ref = oracle.decode_static(case.lgd.numpy(), K, ref_pool["target"], ref_pool["scale"])
+    yref = oracle.moe_apply(A(case.xd), A(case.wg), A(case.wu), A(case.wd), ref["ids"], ref["w"], N, n_shared)
+    ws = case.workspace(B, K)
+    y = torch.full((B, cfg.hidden), float("nan"), dtype=torch.bfloat16, device=dev)
+    meta = dict(ids=torch.full((B, K), -7, dtype=torch.int32, device=dev),
+                w=torch.full((B, K), float("nan"), dtype=torch.float32, device=dev),
+                pool_ids=torch.full((M,), -7, dtype=torch.int32, device=dev))
+    for _ in range(2):
+        ex.exfold_moe_decode_static(case.layer, case.d_xd, case.d_lgd, case.d_wg, case.d_wu, case.d_wd, sp, y, ws,
+                                    meta=meta)
+        assert ex.exfold_device_status(ws) == 0
+        assert np.array_equal(meta["ids"].cpu().numpy(), ref["ids"])
+        np.testing.assert_allclose(meta["w"].cpu().numpy(), ref["w"], rtol=1e-6, atol=1e-7)
+        assert np.array_equal(meta["pool_ids"].cpu().numpy(), ref_pool["pool_ids"])
+        check_output(y.float().cpu().numpy(), yref, "bf16")
+
+
 def test_results_are_reproducible_and_meta_is_optional():
     case = Case(small_bf16())
     a = case.run_prefill(2)
