@@ -57,7 +57,7 @@ void prof_reset() {
 struct Plan {
     size_t status, ids, w, omit_src, omit_tgt, block_hist, offsets, work_start, totals, perm, row_tok, row_w,
         row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
-        xs, H, y32, out, grp_tiles, total;
+        xs, H, y32, out, grp_tiles, obuf, inv_pos, total;
 };
 
 bool valid_layer(const exfold_layer* l) {
@@ -93,6 +93,7 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
     p.work_start = take((G + 2) * 4);
     p.totals = take(16);
     p.perm = take(Rm * 4);
+    p.inv_pos = take(Rm * 4);
     p.row_tok = take(Rtot * 4);
     p.row_w = take(Rtot * 4);
     p.row_exp = take(Rtot * 4);
@@ -116,8 +117,9 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
         a = align_up(Rtot * (size_t)l.hidden * 2, 1024);
         p.H = p.big + a;
         a += align_up(Rtot * (size_t)l.inter * 2, 1024);
-        p.y32 = p.big + a;
-        a += align_up((size_t)Tm * l.hidden * 4, 1024);
+        p.y32 = p.big + a;  // decode: fp32 accumulator [B][d]; prefill: per-route bf16 outputs O [Rtot][d]
+        p.obuf = p.y32;
+        a += align_up(std::max((size_t)Tm * l.hidden * 4, Rtot * (size_t)l.hidden * 2), 1024);
     }
     p.out = p.big;
     size_t b = align_up(Rtot * (size_t)l.hidden * 4, 1024);
@@ -320,7 +322,7 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     cp.x = x; cp.xs = bf16 ? at<char>(ws, pl.xs) : nullptr;
     cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
     cp.row_w = at<float>(ws, pl.row_w); cp.row_exp = at<int32_t>(ws, pl.row_exp);
-    cp.y32 = (bf16 && !direct) ? at<float>(ws, pl.y32) : nullptr; cp.d = d;
+    cp.inv_pos = at<int32_t>(ws, pl.inv_pos);
     { ProfScope ps(2, s); EXFOLD_CUDA(launch_prefill_scatter(cp, s)); }
 
     if (bf16) {
@@ -334,11 +336,18 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
         int grid1 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
         { ProfScope ps(3, s); EXFOLD_CUDA(launch_grouped_gemm1(g, grid1, s)); }
         g.tm_a = tm_h; g.tm_b0 = tm_wd; g.n_ntiles = (d + 255) / 256;
-        g.y32 = direct ? nullptr : at<float>(ws, pl.y32);
-        g.y = reinterpret_cast<__nv_bfloat16*>(y);
+        // K' = 1 without a shared expert: every token is written once, straight into y. Otherwise each
+        // route's weighted output goes to O (bf16, sorted rows) and the combine kernel sums per token.
+        g.y32 = nullptr;
+        g.y = direct ? reinterpret_cast<__nv_bfloat16*>(y) : at<__nv_bfloat16>(ws, pl.obuf);
+        g.store_rows = direct ? 0 : 1;
         int grid2 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
         { ProfScope ps(4, s); EXFOLD_CUDA(launch_grouped_gemm2(g, grid2, s)); }
-        if (!direct) { ProfScope ps(5, s); EXFOLD_CUDA(launch_convert_bf16(at<float>(ws, pl.y32), T * d, y, s)); }
+        if (!direct) {
+            ProfScope ps(5, s);
+            EXFOLD_CUDA(launch_combine_rows(at<__nv_bfloat16>(ws, pl.obuf), cp.inv_pos, T, Kp, d, l.n_shared,
+                                            reinterpret_cast<__nv_bfloat16*>(y), s));
+        }
     } else {
         SimtFfnParams fp{};
         fp.x = x; fp.wg = w_gate; fp.wu = w_up; fp.wd = w_down; fp.dtype = l.dtype; fp.d = d; fp.I = I;
@@ -430,7 +439,7 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
         const int64_t items1 = (int64_t)max_groups * tiles_per_group * g.n_ntiles;
         { ProfScope ps(8, s); EXFOLD_CUDA(launch_grouped_gemm1(g, (int)std::min<int64_t>(sms, items1), s)); }
         g.tm_a = tm_h; g.tm_b0 = tm_wd; g.n_ntiles = (d + 255) / 256;
-        g.y32 = at<float>(ws, pl.y32); g.y = reinterpret_cast<__nv_bfloat16*>(y);
+        g.y32 = at<float>(ws, pl.y32); g.y = reinterpret_cast<__nv_bfloat16*>(y); g.store_rows = 0;
         // split K so that every SM streams a share of W_down even with few (expert, column tile) items
         const int nkb2 = I / 64;
         const int64_t base_items = (int64_t)max_groups * tiles_per_group * g.n_ntiles;

@@ -123,8 +123,7 @@ struct PrefillScatterParams {
     int32_t* row_tok;   // [R + T*n_shared]
     float* row_w;       // [R + T*n_shared]
     int32_t* row_exp;   // [R + T*n_shared]
-    float* y32;         // fp32 accumulator [T][d] to clear (null: nothing to clear)
-    int d;
+    int32_t* inv_pos;   // [R] sorted row of each route (inverse of perm); may be null
 };
 
 cudaError_t launch_prefill_route(const PrefillRouteParams& p, cudaStream_t s);
@@ -183,6 +182,9 @@ cudaError_t launch_simt_ffn(const SimtFfnParams& p, cudaStream_t s);
 cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, int Kr, int d, int n_shared,
                                   void* y, int dtype, cudaStream_t s);
 cudaError_t launch_convert_bf16(const float* y32, int64_t n, void* y, cudaStream_t s);
+// y[i] = sum_j O[inv_pos[i*Kr+j]] (+ O[R+i] for the shared expert), fp32 sum in slot order, bf16 out
+cudaError_t launch_combine_rows(const __nv_bfloat16* O, const int32_t* inv_pos, int64_t T, int Kr, int d,
+                                int n_shared, __nv_bfloat16* y, cudaStream_t s);
 
 // ---------------------------------------------------------------- calibration
 struct CalibStatsParams {
@@ -222,8 +224,9 @@ struct GroupedGemmParams {
     __nv_bfloat16* H;           // GEMM-1 out [Rtot][I]
     const int32_t* row_tok;     // GEMM-2
     const float* row_w;         // GEMM-2
-    float* y32;                 // GEMM-2 accumulate target (null: direct bf16 store)
-    __nv_bfloat16* y;           // GEMM-2 direct target
+    float* y32;                 // GEMM-2 accumulate target (null: bf16 store into y)
+    __nv_bfloat16* y;           // GEMM-2 bf16 target: row = token (store_rows == 0) or the sorted row itself
+    int store_rows;             // 1: y is the per-route buffer O[row][d] that the combine kernel sums
     DeviceStatus* status;
 };
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s);

@@ -84,6 +84,36 @@ __global__ void combine_routes_kernel(const float* __restrict__ out, const float
     }
 }
 
+// Eq. 4's weighted sum for the tensor-core path: GEMM-2 stored w~ * E(x) per route in bf16, sorted by
+// expert; a token's routes are found through the inverse permutation and summed in fp32, slot order.
+__global__ void __launch_bounds__(256) combine_rows_kernel(const __nv_bfloat16* __restrict__ O,
+                                                           const int32_t* __restrict__ inv_pos, int64_t Tn, int Kr, int d,
+                                                           int n_shared, __nv_bfloat16* __restrict__ y) {
+    const int64_t i = blockIdx.x;
+    grid_dep_launch();
+    grid_dep_wait();
+    for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int j = 0; j <= Kr; ++j) {
+            if (j == Kr && !n_shared) break;
+            const int64_t row = j < Kr ? (int64_t)inv_pos[i * Kr + j] : Tn * Kr + i;
+            const uint4 v = *reinterpret_cast<const uint4*>(O + row * d + c);
+            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float2 f = __bfloat1622float2(h2[u]);
+                acc[2 * u] += f.x;
+                acc[2 * u + 1] += f.y;
+            }
+        }
+        uint4 o;
+        __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) o2[u] = __floats2bfloat162_rn(acc[2 * u], acc[2 * u + 1]);
+        *reinterpret_cast<uint4*>(y + i * d + c) = o;
+    }
+}
+
 __global__ void convert_bf16_kernel(const float4* __restrict__ src, int64_t n4, uint2* __restrict__ dst) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -127,6 +157,12 @@ cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, i
                           reinterpret_cast<__nv_bfloat16*>(y));
     return launch_pdl(combine_routes_kernel<float>, (unsigned)T, 256, 0, s, out, w, T, Kr, d, n_shared,
                       reinterpret_cast<float*>(y));
+}
+
+cudaError_t launch_combine_rows(const __nv_bfloat16* O, const int32_t* inv_pos, int64_t T, int Kr, int d,
+                                int n_shared, __nv_bfloat16* y, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    return launch_pdl(combine_rows_kernel, (unsigned)T, 256, 0, s, O, inv_pos, T, Kr, d, n_shared, y);
 }
 
 cudaError_t launch_convert_bf16(const float* y32, int64_t n, void* y, cudaStream_t s) {

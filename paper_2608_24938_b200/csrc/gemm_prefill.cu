@@ -294,7 +294,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
 #pragma unroll
                             for (int j = 0; j < 16; ++j)
                                 pk[j] = pack_bf16(wv * __uint_as_float(v[2 * j]), wv * __uint_as_float(v[2 * j + 1]));
-                            uint4* dst = reinterpret_cast<uint4*>(p.y + (int64_t)tok * p.d + col0);
+                            const int64_t drow = p.store_rows ? grow : (int64_t)tok;
+                            uint4* dst = reinterpret_cast<uint4*>(p.y + drow * p.d + col0);
 #pragma unroll
                             for (int j = 0; j < 4; ++j)
                                 dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);

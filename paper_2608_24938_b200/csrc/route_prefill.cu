@@ -9,7 +9,7 @@
 //                  blocks; block 0 also publishes offsets and the row-tile prefix for the GEMM
 //                  work list), then ranks its routes in (token, slot) order, so the permutation
 //                  is the stable sort by expert and is bit-reproducible; it also gathers the
-//                  token rows into sorted order and clears the fp32 accumulator.
+//                  token rows into sorted order.
 #include "common.cuh"
 
 namespace exfold {
@@ -155,11 +155,6 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_scatter_kernel(PrefillS
     const int64_t r0 = tok0 * Kp;
     grid_dep_launch();
     grid_dep_wait();
-    if (p.y32 != nullptr) {  // clear this block's rows of the fp32 accumulator
-        float4* z = reinterpret_cast<float4*>(p.y32 + (size_t)tok0 * p.d);
-        const int n4 = ntok * p.d / 4;
-        for (int c = threadIdx.x; c < n4; c += blockDim.x) z[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
     // Every block derives its own bases from the per-block histograms (a few KB, L2-resident): the
     // first sorted position of expert e for this block is (rows of experts < e) + (rows of e in
     // earlier blocks). No single-CTA scan kernel sits between routing and the GEMMs.
@@ -217,6 +212,7 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_scatter_kernel(PrefillS
         int q = pos[r];
         int64_t route = r0 + r;
         p.perm[q] = (int32_t)route;
+        if (p.inv_pos != nullptr) p.inv_pos[route] = q;
         p.row_tok[q] = (int32_t)(route / Kp);
         p.row_w[q] = p.w[route];
         p.row_exp[q] = p.ids[route];
