@@ -138,6 +138,22 @@ def oracle_decode_run(cfg, inp, M):
     return dict(dec=dec, y=y, seconds=time.perf_counter() - t0)
 
 
+def max_over_ranks(values, world, device="cpu"):
+    """Element-wise MAX of a list of floats over all ranks (the slowest rank defines the job's time)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_tokens_per_s(tokens_per_rank, world, ms):
+    """Whole-job throughput of `world` independent replicas that each process tokens_per_rank tokens in ms."""
+    return world * tokens_per_rank / (ms * 1e-3)
+
+
 def rel_err(y, ref):
     return float(np.abs(y - ref).max() / np.abs(ref).max()), float(np.linalg.norm(y - ref) / np.linalg.norm(ref))
 
@@ -239,10 +255,7 @@ def run_ours(args, rank, world):
     dec_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))
     pre_min = float(np.min([e[0].elapsed_time(e[1]) for e in ev]))
     dec_min = float(np.min([e[2].elapsed_time(e[3]) for e in ev]))
-    if world > 1:
-        t = torch.tensor([pre_ms, dec_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        pre_ms, dec_ms = float(t[0]), float(t[1])
+    pre_ms, dec_ms = max_over_ranks([pre_ms, dec_ms], world, dev)
 
     # ---- per-kernel durations (CUDA events recorded by the library around each launch)
     ex.exfold_profile_enable(True)
@@ -282,10 +295,7 @@ def run_ours(args, rank, world):
         torch.cuda.synchronize()
     e2e_pre = float(np.mean([e[0].elapsed_time(e[1]) for e in ee]))
     e2e_dec = float(np.mean([e[2].elapsed_time(e[3]) for e in ee]))
-    if world > 1:
-        t = torch.tensor([e2e_pre, e2e_dec], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_pre, e2e_dec = float(t[0]), float(t[1])
+    e2e_pre, e2e_dec = max_over_ranks([e2e_pre, e2e_dec], world, dev)
     el = 2 if cfg.dtype == "bf16" else 4
     h2d = T * d * el + T * N * 4 + B * d * el + B * N * 4
     d2h = T * d * el + B * d * el
@@ -298,7 +308,7 @@ def run_ours(args, rank, world):
     gateup_bytes = pool_bytes * 2.0 / 3.0
     out = {
         "metric": "folded-MoE-layer prefill tokens/s (decode us/layer and roofline fractions alongside)",
-        "value": world * T / (pre_ms * 1e-3),
+        "value": job_tokens_per_s(T, world, pre_ms),
         "unit": "tokens/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": pre_ms + dec_ms,
@@ -318,7 +328,7 @@ def run_ours(args, rank, world):
         "kernels_ms": kern,
         "gpu_launches": int(launches),
         "clocks": sampler.summary(),
-        "e2e": {"value": world * T / (e2e_pre * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
+        "e2e": {"value": job_tokens_per_s(T, world, e2e_pre), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
                 "d2h_bytes_per_step": int(d2h), "prefill_ms": e2e_pre, "decode_us": e2e_dec * 1e3},
         "peaks": {"source": peak_src, **peaks},
         "wall_s_timed_region": wall,

@@ -218,6 +218,25 @@ def test_results_are_reproducible_and_meta_is_optional():
     np.testing.assert_allclose(d2["y"], d1["y"], rtol=0, atol=2e-2 * np.abs(d1["y"]).max())
 
 
+def test_device_status_record_is_decoded_and_cleared():
+    """The status record at the start of the workspace: a code written there (here from the host, never
+    by faulting a kernel) is reported once by exfold_device_status and cleared; every call clears it first."""
+    case = Case(small_bf16())
+    ex = case.ex
+    ws = case.workspace(case.T, 2)
+    ws[:256].zero_()
+    assert ex.exfold_device_status(ws) == ex.EXFOLD_OK
+    ws[:4].copy_(torch.tensor([ex.EXFOLD_ERR_DEVICE_TIMEOUT], dtype=torch.int32).view(torch.uint8))
+    assert ex.exfold_device_status(ws) == ex.EXFOLD_ERR_DEVICE_TIMEOUT
+    assert ex.exfold_device_status(ws) == ex.EXFOLD_OK
+    ws[:4].copy_(torch.tensor([-77], dtype=torch.int32).view(torch.uint8))      # unknown code
+    assert ex.exfold_device_status(ws) == ex.EXFOLD_ERR_CUDA
+    ws[:4].copy_(torch.tensor([ex.EXFOLD_ERR_DEVICE_TIMEOUT], dtype=torch.int32).view(torch.uint8))
+    y = torch.empty((case.T, case.cfg.hidden), dtype=torch.bfloat16, device=case.dev)
+    ex.exfold_moe_prefill(case.layer, case.d_x, case.d_lg, case.d_wg, case.d_wu, case.d_wd, case.tables, 2, y, ws)
+    assert ex.exfold_device_status(ws) == ex.EXFOLD_OK    # a stale code does not survive the next call
+
+
 def test_host_buffer_entry_points():
     case = Case(small_bf16())
     ex, cfg = case.ex, case.cfg
