@@ -329,7 +329,8 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
         GroupedGemmParams g{};
         g.tm_a = tm_xs; g.tm_a2 = tm_x; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu;
         g.offsets = cp.offsets; g.work_start = cp.work_start; g.G = G; g.n_routed = N; g.R = (int)R;
-        g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.grp_expert = nullptr; g.n_groups_dev = nullptr;
+        g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.a_rows = kTileM;
+        g.grp_expert = nullptr; g.n_groups_dev = nullptr;
         g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = cp.row_tok; g.row_w = cp.row_w;
         g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
         const int64_t max_tiles = Rtot / kTileM + G;
@@ -389,13 +390,15 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
     const bool bf16 = l.dtype == EXFOLD_BF16;
     const int max_rows = (int)(B * K + B * l.n_shared);
+    // a group has at most B rows: the token box of the GEMMs needs only that many (multiple of 32, <= 128)
+    const int a_rows = (int)std::min<int64_t>(kTileM, (B + 31) / 32 * 32);
 
     CUtensorMap tm_xs, tm_wg, tm_wu, tm_h, tm_wd;
     if (bf16) {
         const uint64_t E = (uint64_t)G;
-        bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)max_rows, d, 128) &&
+        bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)max_rows, d, a_rows) &&
                   make_tmap(&tm_wg, w_gate, E * I, d, 128) && make_tmap(&tm_wu, w_up, E * I, d, 128) &&
-                  make_tmap(&tm_h, at<char>(ws, pl.H), (uint64_t)max_rows, I, 128) &&
+                  make_tmap(&tm_h, at<char>(ws, pl.H), (uint64_t)max_rows, I, a_rows) &&
                   make_tmap(&tm_wd, w_down, E * d, I, 256);
         if (!ok) return EXFOLD_ERR_CUDA;
     }
@@ -432,7 +435,7 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
         GroupedGemmParams g{};
         g.tm_a = tm_xs; g.tm_a2 = tm_xs; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu;
         g.offsets = rp.grp_off; g.work_start = rp.grp_tiles; g.G = max_groups; g.n_routed = 0x7fffffff;
-        g.R = max_rows; g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1;
+        g.R = max_rows; g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.a_rows = a_rows;
         g.grp_expert = rp.grp_expert; g.n_groups_dev = rp.n_groups;
         g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = rp.row_tok; g.row_w = rp.row_w;
         g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);

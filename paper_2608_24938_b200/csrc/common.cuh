@@ -218,6 +218,7 @@ struct GroupedGemmParams {
     int d, I;
     int n_ntiles;               // column tiles
     int ksplit;                 // GEMM-2: K parts per tile (> 1 only with the y32 reduction epilogue)
+    int a_rows;                 // decode: rows of the A (token) box, a multiple of 32 <= 128; prefill: 128
     const int32_t* grp_expert;  // [G] expert whose weights group g uses (null: g itself)
     const int32_t* n_groups_dev;  // device-side group count (null: G)
     // epilogues

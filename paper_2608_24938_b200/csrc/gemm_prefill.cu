@@ -23,6 +23,7 @@ namespace {
 
 constexpr int kBK = 64;                       // K elements per stage: 128 bytes = one swizzle row
 constexpr int kStages = 4;
+constexpr int kMaxStages = 6;  // decode loads a shorter A box per stage and fits more stages
 constexpr int kATileBytes = kTileM * kBK * 2;  // 16 KB
 constexpr int kBTileBytes = 256 * kBK * 2;     // 32 KB
 constexpr int kStageBytes = kATileBytes + kBTileBytes;
@@ -71,8 +72,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 template <int MODE, bool DEC>
 __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __grid_constant__ GroupedGemmParams p) {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[kStages];
-    __shared__ __align__(8) uint64_t empty_bar[kStages];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
     __shared__ __align__(8) uint64_t tfull_bar[2];
     __shared__ __align__(8) uint64_t tempty_bar[2];
     __shared__ uint32_t tmem_base_s;
@@ -98,7 +99,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
             ptx::prefetch_tmap(&p.tm_a2);
             ptx::prefetch_tmap(&p.tm_b1);
         }
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kMaxStages; ++s) {
             ptx::mbar_init(&full_bar[s], 1);
             ptx::mbar_init(&empty_bar[s], 1);
         }
@@ -140,6 +141,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     const int w_stride = eff_grid > 0 ? eff_grid : 1;
     const int nkb = (MODE == 0 ? p.d : p.I) / kBK;
     const int kb_per = (nkb + ks - 1) / ks;
+    // Stage geometry. Prefill: 16 KB A + 32 KB B, 4 stages (compile-time). Decode: the A box has only
+    // a_rows rows (the rest of the 128-row MMA operand is whatever follows in shared memory: those
+    // accumulator rows are masked), so a stage is smaller and more stages of weights are in flight.
+    const int a_bytes = DEC ? p.a_rows * 128 : kATileBytes;
+    const int stage_bytes = DEC ? a_bytes + kBTileBytes : kStageBytes;
+    const int stages = DEC ? min(kMaxStages, (kStages * kStageBytes - (kATileBytes - a_bytes)) / stage_bytes) : kStages;
     volatile int* abort_flag = &abort_s;
     if (threadIdx.x == 0) EXFOLD_TRACE_SET(kTr, 1, ptx::globaltimer_ns());
 
@@ -164,13 +171,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                         ok = false;
                         break;
                     }
-                    unsigned char* a_dst = tiles + stage * kStageBytes;
-                    unsigned char* b_dst = a_dst + kATileBytes;
-                    ptx::mbar_expect_tx(&full_bar[stage], kStageBytes);
+                    unsigned char* a_dst = tiles + stage * stage_bytes;
+                    unsigned char* b_dst = a_dst + a_bytes;
+                    ptx::mbar_expect_tx(&full_bar[stage], stage_bytes);
                     ptx::tma_load_2d(a_dst, tma_a, &full_bar[stage], kb * kBK, arow);
                     ptx::tma_load_2d(b_dst, &p.tm_b0, &full_bar[stage], kb * kBK, brow);
                     if (MODE == 0) ptx::tma_load_2d(b_dst + 128 * 128, &p.tm_b1, &full_bar[stage], kb * kBK, brow);
-                    if (++stage == kStages) {
+                    if (++stage == stages) {
                         stage = 0;
                         phase ^= 1;
                     }
@@ -203,14 +210,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                         break;
                     }
                     ptx::tc_fence_after();
-                    const uint32_t a_addr = ptx::smem_u32(tiles + stage * kStageBytes);
+                    const uint32_t a_addr = ptx::smem_u32(tiles + stage * stage_bytes);
                     const uint64_t adesc = ptx::make_kmajor_sw128_desc(a_addr);
-                    const uint64_t bdesc = ptx::make_kmajor_sw128_desc(a_addr + kATileBytes);
+                    const uint64_t bdesc = ptx::make_kmajor_sw128_desc(a_addr + a_bytes);
 #pragma unroll
                     for (int k = 0; k < kBK / 16; ++k)
                         ptx::umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
                     ptx::umma_commit(&empty_bar[stage]);
-                    if (++stage == kStages) {
+                    if (++stage == stages) {
                         stage = 0;
                         phase ^= 1;
                     }
