@@ -373,6 +373,78 @@ int orc_prefill_fold(const float *logits, int64_t T, int N, int K, int Kp, const
 }
 
 /*
+ * Prefill folding with the safeguards of the cross-model sections:
+ *  - loss threshold (Qwen3.5 configuration): directed pairs whose calibrated loss exceeds
+ *    loss_thr are excluded from target assignment; an omitted route with no admissible target
+ *    is dropped (reading: the paper does not say);
+ *  - rescale: after folding, the retained weights of a token are scaled by
+ *    (sum of the original K routed weights) / (sum of the folded weights), so the original
+ *    routed-weight sum is preserved (skipped when the folded sum is not positive: reading);
+ *  - confidence split (DeepSeek-V4 appendix): with c_s = clip(1 - l_{s->t*}, 0, 1) for the
+ *    minimum-loss target t*, the part w_s c_s S[s][t*] is folded onto t* and the rest
+ *    w_s (1 - c_s) is spread over the retained routes in proportion to their original
+ *    router weights.
+ * loss_thr = +inf, rescale = 0, confidence = 0 is plain Eq. 13.
+ */
+int orc_prefill_fold_safe(const float *logits, int64_t T, int N, int K, int Kp, const float *S,
+                          const float *L, const float *lnh, double loss_thr, int rescale,
+                          int confidence, int32_t *ids_out, float *w_out, int32_t *omit_src,
+                          int32_t *omit_tgt)
+{
+    if (K < 1 || K > 64 || K > N || Kp < 1 || Kp > K) return -1;
+    int Ko = K - Kp;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < T; ++i) {
+        int32_t ids[64], kept[64], adm[64];
+        double w[64], wt[64], w0[64];
+        int order[64];
+        const float *r = logits + i * N;
+        gate_token(r, N, K, ids, w);
+        prefill_select(r, ids, K, lnh, order);
+        double kept_sum = 0.0, all_sum = 0.0;
+        for (int k = 0; k < K; ++k) all_sum += w[k];
+        for (int j = 0; j < Kp; ++j) {
+            kept[j] = ids[order[j]];
+            wt[j] = w0[j] = w[order[j]];
+            kept_sum += w0[j];
+        }
+        for (int o = 0; o < Ko; ++o) {
+            int slot = order[Kp + o];
+            int s = ids[slot];
+            int na = 0;
+            for (int j = 0; j < Kp; ++j)
+                if (!((double)L[(size_t)s * N + kept[j]] > loss_thr)) adm[na++] = kept[j];
+            int t = na ? argmin_loss(L, N, s, adm, na) : -1;
+            if (t >= 0) {
+                double c = 1.0;
+                if (confidence) {
+                    c = 1.0 - (double)L[(size_t)s * N + t];
+                    if (c < 0.0) c = 0.0;
+                    if (c > 1.0) c = 1.0;
+                }
+                for (int j = 0; j < Kp; ++j) {
+                    if (kept[j] == t) wt[j] += w[slot] * c * (double)S[(size_t)s * N + t];
+                    if (confidence) wt[j] += w[slot] * (1.0 - c) * (w0[j] / kept_sum);
+                }
+            }
+            if (omit_src) omit_src[i * Ko + o] = s;
+            if (omit_tgt) omit_tgt[i * Ko + o] = t;
+        }
+        if (rescale) {
+            double fs = 0.0;
+            for (int j = 0; j < Kp; ++j) fs += wt[j];
+            if (fs > 0.0)
+                for (int j = 0; j < Kp; ++j) wt[j] *= all_sum / fs;
+        }
+        for (int j = 0; j < Kp; ++j) {
+            ids_out[i * Kp + j] = kept[j];
+            w_out[i * Kp + j] = (float)wt[j];
+        }
+    }
+    return 0;
+}
+
+/*
  * Eq. 4 written out for prefill: run every one of the token's K experts' targets and
  * scale: y = sum_{t kept} a_t E_t(x) + sum_{s omitted} a_s S[s][t_s] E_{t_s}(x) (+ shared).
  * Each term evaluates its expert anew; nothing is coalesced.

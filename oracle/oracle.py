@@ -227,3 +227,20 @@ def decode_static(logits, K: int, target, scale):
     rc = _L().orc_decode_static(_p(logits), C.c_int64(B), N, K, _p(target), _p(scale), _p(ids), _p(w))
     assert rc == 0, rc
     return dict(ids=ids, w=w)
+
+
+def prefill_fold_safe(logits, K: int, Kp: int, S, L, lnh, loss_thr: float = float("inf"), rescale: bool = False,
+                      confidence: bool = False):
+    """Prefill folding with the loss-threshold / rescale / confidence-split safeguards.
+    Returns dict(ids, w, omit_src, omit_tgt); omit_tgt is -1 for a dropped route."""
+    logits = _c(logits, np.float32)
+    S, L, lnh = _c(S, np.float32), _c(L, np.float32), _c(lnh, np.float32)
+    T, N = logits.shape
+    ids = np.empty((T, Kp), np.int32)
+    w = np.empty((T, Kp), np.float32)
+    osrc = np.empty((T, K - Kp), np.int32)
+    otgt = np.empty((T, K - Kp), np.int32)
+    rc = _L().orc_prefill_fold_safe(_p(logits), C.c_int64(T), N, K, Kp, _p(S), _p(L), _p(lnh), C.c_double(loss_thr),
+                                    int(rescale), int(confidence), _p(ids), _p(w), _p(osrc), _p(otgt))
+    assert rc == 0, rc
+    return dict(ids=ids, w=w, omit_src=osrc, omit_tgt=otgt)

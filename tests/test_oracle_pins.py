@@ -238,6 +238,53 @@ def test_decode_pool_invariants_and_listing_semantics():
                 assert scl[s] == S[s, tgt[s]]
 
 
+def test_prefill_safeguards():
+    """Loss threshold, rescale and confidence split, each against its own definition in numpy."""
+    g = np.random.default_rng(17)
+    N, K, Kp = 10, 5, 2
+    lg = g.standard_normal((120, N)).astype(np.float32)
+    S, L, h, lnh = rand_tables(N, 9, unobs=0.1)
+    base = oracle.prefill_fold(lg, K, Kp, S, L, h, lnh)
+    off = oracle.prefill_fold_safe(lg, K, Kp, S, L, lnh)
+    for k in ("ids", "w", "omit_src", "omit_tgt"):
+        assert np.array_equal(off[k], base[k])           # all safeguards off = plain Eq. 13
+    ids, w, w64 = oracle.gate(lg, K)
+    thr = 0.6
+    for rescale, conf in ((False, False), (True, False), (False, True), (True, True)):
+        got = oracle.prefill_fold_safe(lg, K, Kp, S, L, lnh, loss_thr=thr, rescale=rescale, confidence=conf)
+        assert np.array_equal(got["ids"], base["ids"]) and np.array_equal(got["omit_src"], base["omit_src"])
+        for i in range(lg.shape[0]):
+            kept = got["ids"][i].tolist()
+            wk = {e: float(w64[i][list(ids[i]).index(e)]) for e in ids[i]}
+            wt = {t: wk[t] for t in kept}
+            ksum = sum(wk[t] for t in kept)
+            for s, t in zip(got["omit_src"][i], got["omit_tgt"][i]):
+                adm = sorted(c for c in kept if not (L[s, c] > thr))
+                if not adm:
+                    assert t == -1
+                    continue
+                assert t == adm[int(np.argmin([L[s, c] for c in adm]))]
+                c = float(np.clip(1.0 - np.float64(L[s, t]), 0, 1)) if conf else 1.0
+                wt[t] += wk[s] * c * float(S[s, t])
+                if conf:
+                    for t2 in kept:
+                        wt[t2] += wk[s] * (1 - c) * wk[t2] / ksum
+            if rescale and sum(wt.values()) > 0:
+                f = 1.0 / sum(wt.values())                 # the K routed weights sum to 1
+                wt = {t: v * f for t, v in wt.items()}
+            np.testing.assert_allclose(got["w"][i], [wt[t] for t in kept], rtol=1e-6, atol=1e-7)
+            if rescale and sum(wt.values()) > 0:
+                np.testing.assert_allclose(got["w"][i].astype(np.float64).sum(), 1.0, atol=1e-6)
+    # confidence split with S == 1: nothing is lost whatever the losses are
+    S1 = np.ones((N, N), np.float32)
+    got = oracle.prefill_fold_safe(lg, K, Kp, S1, L, lnh, confidence=True)
+    np.testing.assert_allclose(got["w"].astype(np.float64).sum(1), 1.0, atol=1e-6)
+    # threshold below every loss: every omitted route is dropped; rescaling restores the sum
+    got = oracle.prefill_fold_safe(lg, K, Kp, S, L, lnh, loss_thr=-1.0, rescale=True)
+    assert (got["omit_tgt"] == -1).all()
+    np.testing.assert_allclose(got["w"].astype(np.float64).sum(1), 1.0, atol=1e-6)
+
+
 def test_static_pool_and_listing_remap():
     """Static pool = the M experts with the largest calibration norm; per-route remap = the appendix
     listing (two table lookups, one multiply per slot); with the dynamic pool's tables the static remap
