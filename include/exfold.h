@@ -141,6 +141,30 @@ int exfold_moe_prefill(const exfold_layer *layer, const void *x, const float *lo
                        const exfold_prefill_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Prefill with the safeguards the paper applies on other model families (cross-model results and
+ * the DeepSeek-V4 appendix). opts == NULL, or all fields at their "off" values, is exfold_moe_prefill.
+ *   loss_threshold    directed pairs with calibrated loss above it are excluded from target
+ *                     assignment (the paper uses 0.99); an omitted route with no admissible target is
+ *                     dropped and reported with omit_tgt = -1. Off: +infinity.
+ *   rescale           != 0: after folding, a token's retained weights are scaled so that they sum
+ *                     to the original sum of its K routed weights (skipped when the folded sum is
+ *                     not positive).
+ *   confidence_split  != 0: with c = clip(1 - L[s][t], 0, 1) for the minimum-loss target t, the part
+ *                     w_s c S[s][t] is folded onto t and w_s (1 - c) is spread over the retained
+ *                     routes in proportion to their original router weights.
+ */
+typedef struct {
+    float loss_threshold;
+    int32_t rescale;
+    int32_t confidence_split;
+} exfold_fold_opts;
+
+int exfold_moe_prefill_ex(const exfold_layer *layer, const void *x, const float *logits, int64_t T,
+                          const void *w_gate, const void *w_up, const void *w_down,
+                          const exfold_tables *tables, int32_t k_pre, const exfold_fold_opts *opts, void *y,
+                          const exfold_prefill_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * Decode: batch-level expert-pool folding (Eq. 11, 12, 14, then Eq. 1 and 4 over the pool
  * only). x [B][d], logits [B][N] -> y [B][d], B <= 256. pool_m = M in [1, N]; the pool is
  * the whole expert union of the batch when that has at most M experts, so pool_m = N is the

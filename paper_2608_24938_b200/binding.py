@@ -29,7 +29,8 @@ EXFOLD_WARN_UNOBSERVED_EXPERT = 1
 EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibrate", "exfold_moe_prefill",
            "exfold_moe_decode", "exfold_moe_prefill_host", "exfold_moe_decode_host", "exfold_device_status",
            "exfold_status_string", "exfold_launch_count", "exfold_profile_enable", "exfold_profile_read",
-           "exfold_moe_decode_noalloc", "exfold_static_pool_build", "exfold_moe_decode_static"]
+           "exfold_moe_decode_noalloc", "exfold_static_pool_build", "exfold_moe_decode_static",
+           "exfold_moe_prefill_ex"]
 PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
                  "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
                  "simt_combine"]
@@ -57,6 +58,10 @@ class exfold_prefill_meta(C.Structure):
 class exfold_decode_meta(C.Structure):
     _fields_ = [("pool_ids", C.c_void_p), ("pool_size", C.c_void_p), ("pool_mask", C.c_void_p), ("ids", C.c_void_p),
                 ("w", C.c_void_p), ("target", C.c_void_p), ("scale", C.c_void_p)]
+
+
+class exfold_fold_opts(C.Structure):
+    _fields_ = [("loss_threshold", C.c_float), ("rescale", C.c_int32), ("confidence_split", C.c_int32)]
 
 
 class exfold_static_pool(C.Structure):
@@ -87,6 +92,9 @@ def _load() -> C.CDLL:
     lib.exfold_moe_decode_noalloc.restype = C.c_int
     lib.exfold_moe_decode_noalloc.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables),
                                               i32, vp, C.POINTER(exfold_decode_meta), vp]
+    lib.exfold_moe_prefill_ex.restype = C.c_int
+    lib.exfold_moe_prefill_ex.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables), i32,
+                                          C.POINTER(exfold_fold_opts), vp, C.POINTER(exfold_prefill_meta), vp, sz, vp]
     lib.exfold_static_pool_build.restype = C.c_int
     lib.exfold_static_pool_build.argtypes = [C.POINTER(exfold_layer), C.POINTER(exfold_tables), i32,
                                              C.POINTER(exfold_static_pool), vp]
@@ -281,4 +289,16 @@ def exfold_moe_decode_static(layer, x, logits, w_gate, w_up, w_down, pool: exfol
                                       _stream(stream))
     if check and rc != 0:
         raise ExfoldError(rc, "exfold_moe_decode_static")
+    return rc
+
+
+def exfold_moe_prefill_ex(layer, x, logits, w_gate, w_up, w_down, tables: exfold_tables, k_pre: int, y, ws,
+                          loss_threshold: float = float("inf"), rescale: bool = False, confidence_split: bool = False,
+                          meta: Optional[dict] = None, stream=None, check: bool = True) -> int:
+    opts = exfold_fold_opts(loss_threshold, int(rescale), int(confidence_split))
+    rc = lib.exfold_moe_prefill_ex(C.byref(layer), _ptr(x), _ptr(logits), x.shape[0], _ptr(w_gate), _ptr(w_up),
+                                   _ptr(w_down), C.byref(tables), k_pre, C.byref(opts), _ptr(y), _prefill_meta(meta),
+                                   _ptr(ws), ws.numel(), _stream(stream))
+    if check and rc != 0:
+        raise ExfoldError(rc, "exfold_moe_prefill_ex")
     return rc

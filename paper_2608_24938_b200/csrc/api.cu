@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cstdio>
+#include <cmath>
 #include <cstring>
 
 #include "common.cuh"
@@ -279,6 +280,14 @@ int exfold_device_status(void* ws, void* cuda_stream) {
 int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* logits, int64_t T, const void* w_gate,
                        const void* w_up, const void* w_down, const exfold_tables* tables, int32_t k_pre, void* y,
                        const exfold_prefill_meta* meta, void* ws, size_t ws_bytes, void* cuda_stream) {
+    return exfold_moe_prefill_ex(layer, x, logits, T, w_gate, w_up, w_down, tables, k_pre, nullptr, y, meta, ws,
+                                 ws_bytes, cuda_stream);
+}
+
+int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float* logits, int64_t T,
+                          const void* w_gate, const void* w_up, const void* w_down, const exfold_tables* tables,
+                          int32_t k_pre, const exfold_fold_opts* opts, void* y, const exfold_prefill_meta* meta,
+                          void* ws, size_t ws_bytes, void* cuda_stream) {
     int rc = check_common(layer, x, logits, T, w_gate, w_up, w_down, tables, y, ws);
     if (rc != EXFOLD_OK) return rc;
     const exfold_layer& l = *layer;
@@ -307,6 +316,9 @@ int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* lo
     PrefillRouteParams rp{};
     rp.logits = logits; rp.S = tables->S; rp.L = tables->L; rp.lnh = tables->lnh;
     rp.T = T; rp.N = N; rp.K = K; rp.Kp = Kp;
+    rp.loss_thr = opts ? opts->loss_threshold : INFINITY;
+    rp.rescale = opts ? opts->rescale : 0;
+    rp.confidence = opts ? opts->confidence_split : 0;
     rp.ids = at<int32_t>(ws, pl.ids); rp.w = at<float>(ws, pl.w);
     rp.omit_src = at<int32_t>(ws, pl.omit_src); rp.omit_tgt = at<int32_t>(ws, pl.omit_tgt);
     rp.block_hist = at<int32_t>(ws, pl.block_hist);
@@ -524,6 +536,7 @@ int exfold_calibrate(const exfold_layer* layer, const void* x_cal, const float* 
         PrefillRouteParams rp{};
         rp.logits = logits_cal; rp.S = out->S; rp.L = out->L; rp.lnh = at<float>(ws, pl.zeros);
         rp.T = m; rp.N = N; rp.K = K; rp.Kp = K; rp.ids = ids; rp.w = at<float>(ws, pl.w);
+        rp.loss_thr = INFINITY;
         rp.omit_src = nullptr; rp.omit_tgt = nullptr; rp.block_hist = at<int32_t>(ws, pl.block_hist);
         rp.status = nullptr;
         EXFOLD_CUDA(launch_prefill_route(rp, s));

@@ -98,6 +98,9 @@ struct PrefillRouteParams {
     const float* lnh;     // [N]
     int64_t T;
     int N, K, Kp;
+    float loss_thr;     // pairs with loss above it are not admissible targets (+inf: off)
+    int rescale;        // keep the original routed-weight sum after folding
+    int confidence;     // confidence-aware split of the folded weight
     int32_t* ids;       // [T][Kp]
     float* w;           // [T][Kp]
     int32_t* omit_src;  // [T][K-Kp] or null

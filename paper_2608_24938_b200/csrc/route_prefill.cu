@@ -104,7 +104,13 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_route_kernel(PrefillRou
         // retained lane t loads L[s][t] and S[s][t] itself (independent loads, all in flight together);
         // a warp arg-min over (loss, id) picks the target, which then adds w_s * S[s][t] to its weight.
         float wt = w;
-        int my_tgt = -1;  // for omitted lanes: the chosen target
+        int my_tgt = -1;  // for omitted lanes: the chosen target (-1: dropped, no admissible target)
+        float kept_sum = 0.f;  // sum of the retained routes' original weights (confidence split only)
+        if (p.confidence) {
+            kept_sum = kept ? w : 0.f;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) kept_sum += __shfl_xor_sync(0xffffffffu, kept_sum, off);
+        }
         for (int rr0 = Kp; rr0 < K; rr0 += 4) {
             int src_lane[4], src_id[4];
             float lv[4], sv[4];
@@ -121,11 +127,31 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_route_kernel(PrefillRou
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 if (rr0 + u >= K) break;  // warp-uniform
-                const int bt = warp_argmin(kept, float_order_key(lv[u]), my_id);
+                const bool adm = kept && !(lv[u] > p.loss_thr);  // loss-threshold safeguard
+                const int bt = warp_argmin(adm, float_order_key(lv[u]), my_id);
                 const float ws = __shfl_sync(0xffffffffu, w, src_lane[u]);
-                if (kept && my_id == bt) wt = __fadd_rn(wt, __fmul_rn(ws, sv[u]));
-                if (lane == src_lane[u]) my_tgt = bt;
+                if (bt != 0x7fffffff) {  // warp-uniform: a target exists
+                    const bool is_t = kept && my_id == bt;
+                    float c = 1.0f;
+                    if (p.confidence) {
+                        const unsigned tm = __ballot_sync(0xffffffffu, is_t);
+                        const float lt = __shfl_sync(0xffffffffu, lv[u], __ffs(tm) - 1);
+                        c = fminf(fmaxf(1.0f - lt, 0.0f), 1.0f);
+                        if (kept) wt = __fadd_rn(wt, ws * (1.0f - c) * (w / kept_sum));
+                    }
+                    if (is_t) wt = __fadd_rn(wt, __fmul_rn(ws * c, sv[u]));
+                }
+                if (lane == src_lane[u]) my_tgt = bt == 0x7fffffff ? -1 : bt;
             }
+        }
+        if (p.rescale) {  // keep the original routed-weight sum
+            float fs = kept ? wt : 0.f, as = has ? w : 0.f;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                fs += __shfl_xor_sync(0xffffffffu, fs, off);
+                as += __shfl_xor_sync(0xffffffffu, as, off);
+            }
+            if (fs > 0.f) wt *= as / fs;
         }
         const int bt = my_tgt;
         if (kept) {

@@ -205,6 +205,29 @@ def test_static_pool_decode(n_shared, M):
         check_output(y.float().cpu().numpy(), yref, "bf16")
 
 
+@pytest.mark.parametrize("thr,rescale,conf", [(0.6, False, False), (0.6, True, False), (float("inf"), False, True),
+                                              (0.5, True, True), (-1.0, True, False)])
+def test_prefill_safeguards(thr, rescale, conf):
+    cfg = small_bf16(n_experts=32, top_k=6, prefill_tokens=500, hidden=128, inter=128)
+    case = Case(cfg)
+    ex, dev, T, K, Kp = case.ex, case.dev, case.T, cfg.top_k, 3
+    S, L, h, lnh = case.np_tables()
+    ref = oracle.prefill_fold_safe(case.lg.numpy(), K, Kp, S, L, lnh, loss_thr=thr, rescale=rescale, confidence=conf)
+    yref = oracle.moe_apply(A(case.x), A(case.wg), A(case.wu), A(case.wd), ref["ids"], ref["w"], cfg.n_experts)
+    ws = case.workspace(T, Kp)
+    y = torch.full((T, cfg.hidden), float("nan"), dtype=torch.bfloat16, device=dev)
+    i32 = dict(dtype=torch.int32, device=dev)
+    meta = dict(ids=torch.full((T, Kp), -7, **i32), w=torch.full((T, Kp), float("nan"), device=dev),
+                omit_src=torch.full((T, K - Kp), -7, **i32), omit_tgt=torch.full((T, K - Kp), -7, **i32))
+    ex.exfold_moe_prefill_ex(case.layer, case.d_x, case.d_lg, case.d_wg, case.d_wu, case.d_wd, case.tables, Kp, y, ws,
+                             loss_threshold=thr, rescale=rescale, confidence_split=conf, meta=meta)
+    assert ex.exfold_device_status(ws) == 0
+    for k in ("ids", "omit_src", "omit_tgt"):
+        assert np.array_equal(meta[k].cpu().numpy(), ref[k]), k
+    np.testing.assert_allclose(meta["w"].cpu().numpy(), ref["w"], rtol=2e-5, atol=2e-5)
+    check_output(y.float().cpu().numpy(), yref, "bf16")
+
+
 def test_results_are_reproducible_and_meta_is_optional():
     case = Case(small_bf16())
     a = case.run_prefill(2)
