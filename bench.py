@@ -35,9 +35,8 @@ import synth_inputs as si  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes measured by ncu (dram__bytes_read.sum + dram__bytes_write.sum) divided by the algorithmic
-# bytes of the same launch, from the reduced-case captures summarised under profiles/
-# (grouped_gemm_mixtral_reduced.md). Traffic grows with the weights, so the full-size figure is this ratio
-# times the full-size algorithmic bytes.
+# bytes of the same launch, from the reduced-case ncu captures whose summaries are under profiles/.
+# Traffic grows with the weights, so the full-size figure is this ratio times the full-size algorithmic bytes.
 NCU_TRAFFIC_RATIO = {"gemm1": 511.3 / 502.3, "decode_gateup": 239.3 / 234.9}
 
 

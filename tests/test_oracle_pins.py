@@ -473,3 +473,26 @@ def test_paper_constants_fixture():
     cal = oracle.calibrate(A(x), lg.numpy(), A(wg), A(wu), A(wd), 5, 2)
     assert (cal["L"][cal["n_obs"] == 0][~np.eye(5, dtype=bool)[cal["n_obs"] == 0]] == np.float32(v["unobserved_loss"])).all()
     assert (np.diag(cal["S"]) == v["self_scalar"]).all()
+
+
+def test_oracle_regression_snapshot():
+    """The oracle on the tiny seeded layer still gives the values stored by tests/golden/make_oracle_golden.py
+    (a guard against accidental changes to the oracle's arithmetic, not a pin of its correctness)."""
+    import importlib.util
+    import json
+    import os
+    here = os.path.join(os.path.dirname(__file__), "golden")
+    spec = importlib.util.spec_from_file_location("make_oracle_golden", os.path.join(here, "make_oracle_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    now = mod.snapshot()
+    with open(os.path.join(here, "oracle_tiny.json")) as f:
+        ref = json.load(f)
+    for k, v in ref.items():
+        if isinstance(v, str):
+            continue
+        if isinstance(v, list) and v and isinstance(v[0], int):
+            assert now[k] == v, k
+        else:
+            np.testing.assert_allclose(np.asarray(now[k], np.float64), np.asarray(v, np.float64), rtol=1e-6, atol=1e-9,
+                                       err_msg=k)
