@@ -325,7 +325,6 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     rp.status = at<DeviceStatus>(ws, pl.status);  // the first kernel of the call clears the status record
     { ProfScope ps(0, s); EXFOLD_CUDA(launch_prefill_route(rp, s)); }
 
-    const int nblk = (int)((T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
     PrefillScatterParams cp{};
     cp.T = T; cp.N = N; cp.n_shared = l.n_shared; cp.Kp = Kp; cp.d_bytes = bf16 ? d * 2 : 0;
     cp.nblk = (int)((T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
