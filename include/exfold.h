@@ -123,6 +123,11 @@ size_t exfold_workspace_bytes(const exfold_layer *layer, int64_t max_tokens, int
  * never observed gets S = 0, L = 1e30; an expert never observed gets the mean h of the
  * others and the call returns EXFOLD_WARN_UNOBSERVED_EXPERT after synchronising the
  * stream (this call is off the serving path and does synchronise).
+ * Expert outputs: fp32 layers use the fp32 SIMT expert kernel; bf16 layers run the same grouped
+ * tensor-core GEMMs as prefill (the SwiGLU activation is rounded to bf16 between the two GEMMs, the
+ * outputs stay fp32), so the tables of a bf16 layer carry that rounding (~1e-3 relative per token).
+ * Workspace: exfold_workspace_bytes(layer, m, K) for mode 0, (layer, m, N) for mode 1 (every expert
+ * runs on every token; m*N <= 2^30). bf16 layers need x_cal and the weights 16-byte aligned.
  */
 int exfold_calibrate(const exfold_layer *layer, const void *x_cal, const float *logits_cal, int64_t m,
                      const void *w_gate, const void *w_up, const void *w_down,

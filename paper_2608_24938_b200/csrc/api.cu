@@ -58,7 +58,7 @@ void prof_reset() {
 struct Plan {
     size_t status, ids, w, omit_src, omit_tgt, block_hist, offsets, work_start, totals, perm, row_tok, row_w,
         row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
-        xs, H, y32, out, grp_tiles, obuf, inv_pos, total;
+        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, total;
 };
 
 bool valid_layer(const exfold_layer* l) {
@@ -109,18 +109,21 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
     p.n_groups = take(16);
     p.zeros = take((size_t)N * 4);
     p.calib = take((size_t)N * N * (3 * 8 + 4) + (size_t)N * (8 + 4) + 256);
+    p.calib_nrm = take(Rm * 8);  // calibration, common-input mode: squared output norms per (token, expert)
     // large buffers: the bf16 pipeline (sorted rows, H, fp32 accumulator) and the SIMT path's
     // per-route outputs are never live at the same time and share one region
     p.big = off;
     size_t a = 0;
     if (l.dtype == EXFOLD_BF16) {
+        // xs and obuf are adjacent: calibration reuses the two together (>= Rtot*d*4 bytes) for the
+        // fp32 per-row expert outputs once GEMM-1 has consumed the gathered rows
         p.xs = p.big;
         a = align_up(Rtot * (size_t)l.hidden * 2, 1024);
-        p.H = p.big + a;
-        a += align_up(Rtot * (size_t)l.inter * 2, 1024);
         p.y32 = p.big + a;  // decode: fp32 accumulator [B][d]; prefill: per-route bf16 outputs O [Rtot][d]
         p.obuf = p.y32;
         a += align_up(std::max((size_t)Tm * l.hidden * 4, Rtot * (size_t)l.hidden * 2), 1024);
+        p.H = p.big + a;
+        a += align_up(Rtot * (size_t)l.inter * 2, 1024);
     }
     p.out = p.big;
     size_t b = align_up(Rtot * (size_t)l.hidden * 4, 1024);
@@ -338,7 +341,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
 
     if (bf16) {
         GroupedGemmParams g{};
-        g.tm_a = tm_xs; g.tm_a2 = tm_x; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu;
+        g.tm_a = tm_xs; g.tm_a2 = tm_x; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu; g.x_rows = (int)T; g.o32 = nullptr;
         g.offsets = cp.offsets; g.work_start = cp.work_start; g.G = G; g.n_routed = N; g.R = (int)R;
         g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.a_rows = kTileM;
         g.grp_expert = nullptr; g.n_groups_dev = nullptr;
@@ -444,7 +447,7 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
         const int tiles_per_group = (int)((B + kTileM - 1) / kTileM);
         const int sms = std::min(sm_count(), kMaxCtas);
         GroupedGemmParams g{};
-        g.tm_a = tm_xs; g.tm_a2 = tm_xs; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu;
+        g.tm_a = tm_xs; g.tm_a2 = tm_xs; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu; g.x_rows = 1; g.o32 = nullptr;
         g.offsets = rp.grp_off; g.work_start = rp.grp_tiles; g.G = max_groups; g.n_routed = 0x7fffffff;
         g.R = max_rows; g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.a_rows = a_rows;
         g.grp_expert = rp.grp_expert; g.n_groups_dev = rp.n_groups;
@@ -542,22 +545,76 @@ int exfold_calibrate(const exfold_layer* layer, const void* x_cal, const float* 
     } else {
         EXFOLD_CUDA(launch_iota_ids(ids, m, N, s));
     }
-    SimtFfnParams fp{};
-    fp.x = x_cal; fp.wg = w_gate; fp.wu = w_up; fp.wd = w_down; fp.dtype = l.dtype; fp.d = d; fp.I = I;
-    fp.T = m; fp.Kr = Ke; fp.n_shared = 0; fp.N = N; fp.ids = ids; fp.out = at<float>(ws, pl.out);
-    EXFOLD_CUDA(launch_simt_ffn(fp, s));
+    const bool tensor_path = l.dtype == EXFOLD_BF16;
+    if (tensor_path && (!aligned16(x_cal) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(w_down)))
+        return EXFOLD_ERR_INVALID_ARG;
+    const int64_t Rc = m * Ke;
+    if (tensor_path && Rc > (int64_t)1 << 30) return EXFOLD_ERR_UNSUPPORTED;
+    CalibStatsParams cs{};
+    if (tensor_path) {
+        // Expert outputs on the tensor cores: rows sorted by expert -> GEMM-1 (SwiGLU, H in bf16) -> GEMM-2
+        // with the raw fp32 accumulators stored per sorted row. Mode 0 sorts the routed rows like prefill;
+        // in mode 1 every expert's rows are the tokens themselves, read from x_cal without a copy.
+        CUtensorMap tm_xs, tm_x, tm_wg, tm_wu, tm_h, tm_wd;
+        const uint64_t E = (uint64_t)N;
+        bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)Rc, d, 128) &&
+                  make_tmap(&tm_x, x_cal, (uint64_t)m, d, 128) && make_tmap(&tm_wg, w_gate, E * I, d, 128) &&
+                  make_tmap(&tm_wu, w_up, E * I, d, 128) && make_tmap(&tm_h, at<char>(ws, pl.H), (uint64_t)Rc, I, 128) &&
+                  make_tmap(&tm_wd, w_down, E * d, I, 256);
+        if (!ok) return EXFOLD_ERR_CUDA;
+        int32_t* offsets = at<int32_t>(ws, pl.offsets);
+        int32_t* work_start = at<int32_t>(ws, pl.work_start);
+        if (opts->mode == 0) {
+            PrefillScatterParams cp{};
+            cp.T = m; cp.N = N; cp.n_shared = 0; cp.Kp = K; cp.d_bytes = d * 2;
+            cp.nblk = (int)((m + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
+            cp.ids = ids; cp.w = at<float>(ws, pl.w); cp.block_hist = at<int32_t>(ws, pl.block_hist);
+            cp.offsets = offsets; cp.work_start = work_start;
+            cp.x = x_cal; cp.xs = at<char>(ws, pl.xs);
+            cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
+            cp.row_w = at<float>(ws, pl.row_w); cp.row_exp = at<int32_t>(ws, pl.row_exp);
+            cp.inv_pos = at<int32_t>(ws, pl.inv_pos);
+            EXFOLD_CUDA(launch_prefill_scatter(cp, s));
+            cs.inv_pos = cp.inv_pos;
+        } else {
+            EXFOLD_CUDA(launch_calib_common_rows(offsets, work_start, m, N, s));
+            cs.inv_pos = nullptr; cs.tok_stride = 1; cs.slot_stride = m;
+        }
+        GroupedGemmParams g{};
+        g.tm_a = tm_xs; g.tm_a2 = tm_x; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu;
+        g.offsets = offsets; g.work_start = work_start; g.G = N;
+        g.n_routed = opts->mode == 0 ? N : 0;  // mode 1: every group reads x_cal directly
+        g.R = 0; g.x_rows = (int)m;
+        g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.a_rows = kTileM;
+        g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = at<int32_t>(ws, pl.row_tok); g.row_w = at<float>(ws, pl.row_w);
+        g.status = at<DeviceStatus>(ws, pl.status);
+        const int64_t max_tiles = Rc / kTileM + N;
+        EXFOLD_CUDA(launch_grouped_gemm1(g, (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles), s));
+        g.tm_a = tm_h; g.tm_b0 = tm_wd; g.n_ntiles = (d + 255) / 256;
+        g.o32 = at<float>(ws, pl.xs);  // spans the xs and obuf regions (GEMM-1 is done with xs)
+        EXFOLD_CUDA(launch_grouped_gemm2(g, (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles), s));
+        cs.out = g.o32;
+    } else {
+        SimtFfnParams fp{};
+        fp.x = x_cal; fp.wg = w_gate; fp.wu = w_up; fp.wd = w_down; fp.dtype = l.dtype; fp.d = d; fp.I = I;
+        fp.T = m; fp.Kr = Ke; fp.n_shared = 0; fp.N = N; fp.ids = ids; fp.out = at<float>(ws, pl.out);
+        EXFOLD_CUDA(launch_simt_ffn(fp, s));
+        cs.out = fp.out; cs.inv_pos = nullptr; cs.tok_stride = Ke; cs.slot_stride = 1;
+    }
 
     char* cb = at<char>(ws, pl.calib);
     const size_t NN = (size_t)N * N;
     EXFOLD_CUDA(cudaMemsetAsync(cb, 0, NN * (3 * 8 + 4) + (size_t)N * (8 + 4) + 256, s));
-    CalibStatsParams cs{};
-    cs.out = fp.out; cs.ids = ids; cs.m = m; cs.Ke = Ke; cs.d = d; cs.N = N;
+    cs.ids = ids; cs.m = m; cs.Ke = Ke; cs.d = d; cs.N = N;
     cs.A = reinterpret_cast<double*>(cb); cs.Bv = cs.A + NN; cs.C = cs.Bv + NN;
     cs.H = cs.C + NN;
     cs.cnt = reinterpret_cast<int32_t*>(cs.H + N);
     cs.hc = cs.cnt + NN;
     int32_t* unobs = cs.hc + N;
-    EXFOLD_CUDA(launch_calib_stats(cs, s));
+    if (opts->mode == 1 && Ke >= 32)  // many experts per token: Gram-product form of the same sums
+        EXFOLD_CUDA(launch_calib_stats_common(cs, at<double>(ws, pl.calib_nrm), sm_count(), s));
+    else
+        EXFOLD_CUDA(launch_calib_stats(cs, s));
     EXFOLD_CUDA(launch_calib_finalize(cs, *opts, out->S, out->L, out->h, out->lnh, out->n_obs, unobs, s));
     int un = 0;
     EXFOLD_CUDA(cudaMemcpyAsync(&un, unobs, 4, cudaMemcpyDeviceToHost, s));

@@ -191,7 +191,10 @@ cudaError_t launch_combine_rows(const __nv_bfloat16* O, const int32_t* inv_pos, 
 
 // ---------------------------------------------------------------- calibration
 struct CalibStatsParams {
-    const float* out;    // [m][Ke][d] expert outputs
+    const float* out;    // expert outputs, one row of d floats per (token, slot)
+    // row of (token i, slot a): inv_pos[i*Ke + a] if inv_pos is set, else i*tok_stride + a*slot_stride
+    const int32_t* inv_pos;
+    int64_t tok_stride, slot_stride;
     const int32_t* ids;  // [m][Ke]
     int64_t m;
     int Ke, d, N;
@@ -203,9 +206,14 @@ struct CalibStatsParams {
     int32_t* hc;   // [N]
 };
 cudaError_t launch_calib_stats(const CalibStatsParams& p, cudaStream_t s);
+// Common-input mode with identity slots (slot a = expert a, inv_pos unused): same sums via per-token Gram
+// products held in registers; nrm is scratch for m*Ke doubles
+cudaError_t launch_calib_stats_common(const CalibStatsParams& p, double* nrm, int sms, cudaStream_t s);
 cudaError_t launch_calib_finalize(const CalibStatsParams& p, const exfold_calib_opts& o, float* S, float* L,
                                   float* h, float* lnh, int32_t* n_obs, int32_t* unobserved, cudaStream_t s);
 cudaError_t launch_iota_ids(int32_t* ids, int64_t m, int N, cudaStream_t s);
+// Common-input calibration on the grouped GEMMs: every expert e owns rows [e*m, (e+1)*m) = all tokens in order
+cudaError_t launch_calib_common_rows(int32_t* offsets, int32_t* work_start, int64_t m, int N, cudaStream_t s);
 
 // ---------------------------------------------------------------- tcgen05 grouped GEMMs (bf16)
 struct GroupedGemmParams {
@@ -231,6 +239,8 @@ struct GroupedGemmParams {
     float* y32;                 // GEMM-2 accumulate target (null: bf16 store into y)
     __nv_bfloat16* y;           // GEMM-2 bf16 target: row = token (store_rows == 0) or the sorted row itself
     int store_rows;             // 1: y is the per-route buffer O[row][d] that the combine kernel sums
+    float* o32;                 // GEMM-2, calibration: unweighted fp32 outputs O32[row][d] (null: the epilogues above)
+    int x_rows;                 // GEMM-1: rows of x; a group that reads x directly starts at row (row0 - R) % x_rows
     DeviceStatus* status;
 };
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s);

@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                 const int expert = DEC ? s_exp[it.g] : it.g;
                 const bool from_x = !DEC && MODE == 0 && expert >= p.n_routed;  // prefill's shared expert reads x directly
                 const CUtensorMap* tma_a = from_x ? &p.tm_a2 : &p.tm_a;
-                const int arow = from_x ? it.row0 - p.R : it.row0;
+                const int arow = from_x ? (it.row0 - p.R) % p.x_rows : it.row0;
                 const int brow = MODE == 0 ? expert * p.I + it.n_idx * 128 : expert * p.d + it.n_idx * 256;
                 for (int kb = kb0; kb < kb1; ++kb) {
                     bool got;
@@ -289,7 +289,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                     ptx::tmem_ld_wait();
                     const int col0 = it.n_idx * 256 + c * 32;
                     if (valid && col0 < p.d) {
-                        if (p.y32 != nullptr) {
+                        if (!DEC && p.o32 != nullptr) {  // calibration: raw fp32 expert outputs by sorted row
+                            float4* dst = reinterpret_cast<float4*>(p.o32 + grow * p.d + col0);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                        } else if (p.y32 != nullptr) {
                             float* dst = p.y32 + (int64_t)tok * p.d + col0;
 #pragma unroll
                             for (int j = 0; j < 8; ++j)

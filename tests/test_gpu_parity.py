@@ -73,6 +73,66 @@ def test_calibrate_matches_oracle(mode):
     assert (np.diag(S.cpu().numpy()) == 1).all() and (np.diag(L.cpu().numpy()) == 0).all()
 
 
+def test_calibrate_common_input_many_experts_fp32():
+    """Common-input mode with N >= 32 takes the Gram-product form of the pair sums; fp32 layer, tight bound."""
+    cfg = si.LayerConfig("f32_many", 40, 0, 96, 64, 2, "f32", 64, (1,), 16, (4,))
+    case = Case(cfg, std=0.05, correlated=0.8)
+    ex, dev = case.ex, case.dev
+    m, N, K = 203, cfg.n_experts, cfg.top_k
+    xc = si.hidden_states(cfg, m, "x_cal")
+    lc = si.router_logits(cfg, m, "logits_cal")
+    ref = oracle.calibrate(A(xc), lc.numpy(), A(case.wg), A(case.wu), A(case.wd), N, K, mode=1)
+    S = torch.full((N, N), float("nan"), device=dev)
+    L, h, lnh = torch.full_like(S, float("nan")), torch.full((N,), float("nan"), device=dev), torch.empty(N, device=dev)
+    n_obs = torch.full((N, N), -1, dtype=torch.int32, device=dev)
+    ws = ex.alloc_workspace(case.layer, m, N)
+    ws.fill_(0xFF)
+    rc = ex.exfold_calibrate(case.layer, xc.to(dev), lc.to(dev), case.d_wg, case.d_wu, case.d_wd,
+                             ex.make_tables(S, L, h, lnh, n_obs), ws, mode=1)
+    assert rc == 0
+    assert np.array_equal(n_obs.cpu().numpy(), ref["n_obs"])
+    np.testing.assert_allclose(S.cpu().numpy(), ref["S"], rtol=2e-5, atol=2e-6)
+    np.testing.assert_allclose(L.cpu().numpy(), ref["L"], rtol=1e-4, atol=2e-5)
+    np.testing.assert_allclose(h.cpu().numpy(), ref["h"], rtol=1e-5)
+
+
+@pytest.mark.parametrize("mode,N", [(0, 16), (1, 16), (1, 40)])
+def test_calibrate_bf16_on_tensor_cores(mode, N):
+    """bf16 layers calibrate through the grouped tcgen05 GEMMs (Eq. 6-9 on fp32 outputs, H rounded to bf16).
+
+    Tolerance: rounding H to bf16 perturbs every expert output by ~2^-9/sqrt(3) of its norm in a random
+    direction, so per-token inner products move by ~1e-3 relative; the tables average many tokens.
+    700 tokens = several 128-row tiles per expert plus a ragged tail.
+    """
+    cfg = small_bf16(n_experts=N)
+    case = Case(cfg, correlated=0.8)
+    ex, dev = case.ex, case.dev
+    m, K = 700, cfg.top_k
+    xc = si.hidden_states(cfg, m, "x_cal")
+    lc = si.router_logits(cfg, m, "logits_cal")
+    ref = oracle.calibrate(A(xc), lc.numpy(), A(case.wg), A(case.wu), A(case.wd), N, K, mode=mode)
+    S = torch.full((N, N), float("nan"), device=dev)
+    L, h, lnh = torch.full_like(S, float("nan")), torch.full((N,), float("nan"), device=dev), torch.empty(N, device=dev)
+    n_obs = torch.full((N, N), -1, dtype=torch.int32, device=dev)
+    ws = ex.alloc_workspace(case.layer, m, N if mode else K)
+    ws.fill_(0xFF)
+    rc = ex.exfold_calibrate(case.layer, xc.to(dev), lc.to(dev), case.d_wg, case.d_wu, case.d_wd,
+                             ex.make_tables(S, L, h, lnh, n_obs), ws, mode=mode)
+    assert rc == (1 if ref["unobserved"] else 0)
+    assert ex.exfold_device_status(ws) == 0
+    assert np.array_equal(n_obs.cpu().numpy(), ref["n_obs"])
+    Sg, Lg = S.cpu().numpy(), L.cpu().numpy()
+    seen = ref["n_obs"] > 0
+    off = ~np.eye(N, dtype=bool)
+    assert np.abs(ref["S"][off & seen]).mean() > 0.1          # a table worth comparing
+    np.testing.assert_allclose(Sg, ref["S"], rtol=5e-3, atol=5e-3)
+    np.testing.assert_allclose(Lg[seen | ~off], ref["L"][seen | ~off], rtol=5e-3, atol=5e-3)
+    assert (Lg[~seen & off] == np.float32(1e30)).all() and (Sg[~seen & off] == 0).all()
+    np.testing.assert_allclose(h.cpu().numpy(), ref["h"], rtol=3e-3)
+    np.testing.assert_allclose(lnh.cpu().numpy(), ref["lnh"], rtol=0, atol=3e-3)
+    assert (np.diag(Sg) == 1).all() and (np.diag(Lg) == 0).all()
+
+
 # ------------------------------------------------------------------ bf16 tensor-core path
 @pytest.mark.parametrize("Kp", [2, 1, 4])
 def test_bf16_prefill_small(Kp):
