@@ -211,6 +211,24 @@ def test_full_budget_is_the_unfolded_layer():
     check_output(gotd["y"], yd_unf, "bf16")
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_maximum_expert_count_and_top_k(dtype):
+    """N = 256 experts and K = 32 routes per token are the limits of the interface."""
+    cfg = small_bf16(n_experts=256, top_k=32, hidden=128, inter=128, dtype=dtype, prefill_tokens=150,
+                     decode_batch=40, logits="normal")
+    case = Case(cfg)
+    for Kp in (8, 31):
+        got, ref = case.run_prefill(Kp), case.oracle_prefill(Kp)
+        assert ref["mismatch"] == 0
+        check_prefill_meta(got, ref)
+        check_output(got["y"], ref["y"], dtype)
+    for M in (64, 256):
+        got, ref = case.run_decode(M), case.oracle_decode(M)
+        assert ref["min_gap"] > 1e-9
+        check_decode_meta(got, ref, M)
+        check_output(got["y"], ref["y"], dtype)
+
+
 def test_decode_max_batch_and_all_unobserved_row():
     cfg = small_bf16(n_experts=32, top_k=8, decode_batch=256, prefill_tokens=64)
     case = Case(cfg)
