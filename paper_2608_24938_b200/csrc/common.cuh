@@ -108,7 +108,7 @@ struct PrefillRouteParams {
     int32_t* block_hist;  // [nblk][N]
     DeviceStatus* status; // cleared by block 0 (first kernel of a call); may be null
 };
-constexpr int kRouteTokensPerBlock = 64;
+constexpr int kRouteTokensPerBlock = 32;
 constexpr int kRouteThreads = 512;
 
 struct PrefillScatterParams {
