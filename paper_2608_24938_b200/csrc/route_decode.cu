@@ -1,23 +1,29 @@
 // Decode routing: batch-level expert pool (Eq. 11), minimum-loss targets (Eq. 12) and the
-// in-place remap of every routed slot (Eq. 14), in ONE CTA: B*K <= 4096 slots live in
-// shared memory. Also builds the execution lists for the weight-streaming FFN: rows sorted
+// in-place remap of every routed slot (Eq. 14). B*K <= 4096 slots live in the shared memory of one
+// CTA; the per-token Top-K, which is instruction-issue bound on a single SM, is spread over a cluster
+// of 8 CTAs that write their routes and score sums into the first CTA's shared memory and then leave. Also builds the execution lists for the weight-streaming FFN: rows sorted
 // by pool rank, duplicate (token, expert) slots merged ("routes folded into the same target
 // are coalesced before expert computation").
 #include "common.cuh"
 #include "ptx.cuh"
 
+#include <cooperative_groups.h>
+
 namespace exfold {
 
 namespace {
 
+namespace cg = cooperative_groups;
+
 #ifdef EXFOLD_TRACE
-#define DEC_T(slot) if (threadIdx.x == 0) g_trace[2][0][slot] = ptx::globaltimer_ns()
+#define DEC_T(slot) if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[2][0][slot] = ptx::globaltimer_ns()
 #else
 #define DEC_T(slot) ((void)0)
 #endif
 
 constexpr int kDecThreads = 1024;
 constexpr int kDecMaxSlots = 4096;
+constexpr int kDecCluster = 8;  // CTAs that share the Top-K phase
 
 struct DecSmem {
     double w64[kDecMaxSlots];
@@ -42,35 +48,42 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kWarps = kDecThreads / 32;
     const int B = p.B, N = p.N, K = p.K, M = p.M;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank(), nct = (int)cluster.num_blocks();
+    DecSmem* sm0 = rank == 0 ? &sm : cluster.map_shared_rank(&sm, 0);  // the first CTA collects everything
     DEC_T(0);
     grid_dep_launch();
     grid_dep_wait();
     DEC_T(1);
-    if (p.status != nullptr && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
+    if (p.status != nullptr && rank == 0 && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
     // pull the loss and scalar tables towards L2 now; they are needed after the pool is known
     if (p.st_pool == nullptr) {
         const size_t table_bytes = (size_t)N * N * sizeof(float);
-        for (size_t off = (size_t)threadIdx.x * 128; off < table_bytes; off += (size_t)kDecThreads * 128) {
+        for (size_t off = ((size_t)rank * kDecThreads + threadIdx.x) * 128; off < table_bytes;
+             off += (size_t)nct * kDecThreads * 128) {
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(p.L) + off));
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(p.S) + off));
         }
     }
 
-    for (int e = threadIdx.x; e < N; e += kDecThreads) {
-        sm.acc[e] = 0ull;
-        sm.in_union[e] = 0;
-    }
-    __syncthreads();
-    // ---- Eq. 2 per token (warp per token), weights in double; the next token's logits are fetched
-    // while the current one is processed. Each route adds its weight to its expert's fixed-point
-    // accumulator (integer atomics: the sum does not depend on the order of arrival).
+    if (rank == 0)
+        for (int e = threadIdx.x; e < N; e += kDecThreads) {
+            sm.acc[e] = 0ull;
+            sm.in_union[e] = 0;
+        }
+    cluster.sync();
+    // ---- Eq. 2 per token (warp per token, tokens dealt round-robin over the cluster's CTAs), weights in
+    // double; the next token's logits are fetched while the current one is processed. Each route adds its
+    // weight to its expert's fixed-point accumulator in the first CTA (integer atomics: the sum does not
+    // depend on the order of arrival).
+    const int i_first = rank + nct * warp, i_step = nct * kWarps;
     float vn[NPL];
 #pragma unroll
     for (int q = 0; q < NPL; ++q) {
         const int e = lane + 32 * q;
-        vn[q] = (warp < B && e < N) ? p.logits[(size_t)warp * N + e] : -INFINITY;
+        vn[q] = (i_first < B && e < N) ? p.logits[(size_t)i_first * N + e] : -INFINITY;
     }
-    for (int i = warp; i < B; i += kWarps) {
+    for (int i = i_first; i < B; i += i_step) {
         uint32_t key_q[NPL];
         uint32_t used = 0;
 #pragma unroll
@@ -81,7 +94,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
 #pragma unroll
         for (int q = 0; q < NPL; ++q) {
             const int e = lane + 32 * q;
-            vn[q] = (i + kWarps < B && e < N) ? p.logits[(size_t)(i + kWarps) * N + e] : -INFINITY;
+            vn[q] = (i + i_step < B && e < N) ? p.logits[(size_t)(i + i_step) * N + e] : -INFINITY;
         }
         int my_id = -1;
         float my_r = 0.f;
@@ -110,13 +123,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         for (int k = 0; k < K; ++k) sum += __shfl_sync(0xffffffffu, ex, k);  // slot order, like the definition
         if (lane < K) {
             const double wv = ex / sum;
-            sm.ids[i * K + lane] = my_id;
-            sm.w64[i * K + lane] = wv;
-            atomicAdd(&sm.acc[my_id], (unsigned long long)(wv * 9007199254740992.0));  // 2^53
-            sm.in_union[my_id] = 1;
+            sm0->ids[i * K + lane] = my_id;
+            sm0->w64[i * K + lane] = wv;
+            atomicAdd(&sm0->acc[my_id], (unsigned long long)(wv * 9007199254740992.0));  // 2^53
+            sm0->in_union[my_id] = 1;
         }
     }
-    __syncthreads();
+    cluster.sync();  // every CTA's routes and sums have landed in the first CTA
+    if (rank != 0) return;
     DEC_T(2);
 
     const int nslots = B * K;
@@ -385,7 +399,7 @@ cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s) {
     err = cudaFuncSetAttribute(decode_route_kernel<NPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
                                (int)smem);                                                                  \
     if (err != cudaSuccess) return err;                                                                     \
-    err = launch_pdl(decode_route_kernel<NPL>, 1, kDecThreads, smem, s, p);
+    err = launch_pdl_cluster(decode_route_kernel<NPL>, kDecCluster, kDecThreads, smem, kDecCluster, s, p);
     switch (npl) {
         case 1: EXFOLD_DEC_LAUNCH(1) break;
         case 2: EXFOLD_DEC_LAUNCH(2) break;
