@@ -1,7 +1,9 @@
 // Decode routing: batch-level expert pool (Eq. 11), minimum-loss targets (Eq. 12) and the
 // in-place remap of every routed slot (Eq. 14). B*K <= 4096 slots live in the shared memory of one
-// CTA; the per-token Top-K, which is instruction-issue bound on a single SM, is spread over a cluster
-// of 8 CTAs that write their routes and score sums into the first CTA's shared memory and then leave. Also builds the execution lists for the weight-streaming FFN: rows sorted
+// CTA. The kernel runs as one cluster of 8 CTAs, each holding a full copy of that state: the per-token
+// Top-K (instruction-issue bound on a single SM), the target search (each CTA keeps its slice of the
+// loss / scalar table rows in shared memory) and the row lists are dealt over the CTAs and their results
+// broadcast into every copy through distributed shared memory; the cheap steps in between are replicated. Also builds the execution lists for the weight-streaming FFN: rows sorted
 // by pool rank, duplicate (token, expert) slots merged ("routes folded into the same target
 // are coalesced before expert computation").
 #include "common.cuh"
@@ -40,6 +42,7 @@ struct DecSmem {
     int goff[kMaxExperts + 2];
     int P;
 };
+constexpr size_t kDecSmemBytes = (sizeof(DecSmem) + 15) / 16 * 16;  // the table rows follow
 
 template <int NPL>
 __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRouteParams p) {
@@ -50,38 +53,43 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     const int B = p.B, N = p.N, K = p.K, M = p.M;
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank(), nct = (int)cluster.num_blocks();
-    DecSmem* sm0 = rank == 0 ? &sm : cluster.map_shared_rank(&sm, 0);  // the first CTA collects everything
+    // Every CTA keeps a full copy of the small per-batch state; results are broadcast into all copies.
+    DecSmem* peer[kDecCluster];
+#pragma unroll
+    for (int r = 0; r < kDecCluster; ++r) peer[r] = r < nct ? cluster.map_shared_rank(&sm, r) : &sm;
+    const bool is_static = p.st_pool != nullptr;
+    // this CTA's slice of source experts and its rows of the loss / scalar tables (shared memory)
+    const int rows_per = (N + nct - 1) / nct;
+    const int s_lo = min(N, rank * rows_per), s_hi = min(N, s_lo + rows_per);
+    float* tL = reinterpret_cast<float*>(smraw + kDecSmemBytes);
+    float* tS = tL + (size_t)rows_per * N;
     DEC_T(0);
     grid_dep_launch();
     grid_dep_wait();
     DEC_T(1);
     if (p.status != nullptr && rank == 0 && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
-    // pull the loss and scalar tables towards L2 now; they are needed after the pool is known
-    if (p.st_pool == nullptr) {
-        const size_t table_bytes = (size_t)N * N * sizeof(float);
-        for (size_t off = ((size_t)rank * kDecThreads + threadIdx.x) * 128; off < table_bytes;
-             off += (size_t)nct * kDecThreads * 128) {
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(p.L) + off));
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(p.S) + off));
-        }
+    for (int e = threadIdx.x; e < N; e += kDecThreads) {
+        sm.acc[e] = 0ull;
+        sm.in_union[e] = 0;
     }
-
-    if (rank == 0)
-        for (int e = threadIdx.x; e < N; e += kDecThreads) {
-            sm.acc[e] = 0ull;
-            sm.in_union[e] = 0;
-        }
-    cluster.sync();
+    cluster.sync();  // every copy is cleared before any CTA adds to it
     // ---- Eq. 2 per token (warp per token, tokens dealt round-robin over the cluster's CTAs), weights in
-    // double; the next token's logits are fetched while the current one is processed. Each route adds its
-    // weight to its expert's fixed-point accumulator in the first CTA (integer atomics: the sum does not
-    // depend on the order of arrival).
+    // double; the first token's logits are requested before the table rows so that they arrive first.
     const int i_first = rank + nct * warp, i_step = nct * kWarps;
     float vn[NPL];
 #pragma unroll
     for (int q = 0; q < NPL; ++q) {
         const int e = lane + 32 * q;
         vn[q] = (i_first < B && e < N) ? p.logits[(size_t)i_first * N + e] : -INFINITY;
+    }
+    if (!is_static) {  // rows [s_lo, s_hi) of L and S: needed once the pool is known, in flight during the Top-K
+        const int n_el = (s_hi - s_lo) * N;
+        const float* gL = p.L + (size_t)s_lo * N;
+        const float* gS = p.S + (size_t)s_lo * N;
+        for (int idx = threadIdx.x; idx < n_el; idx += kDecThreads) {
+            tL[idx] = __ldg(gL + idx);
+            tS[idx] = __ldg(gS + idx);
+        }
     }
     for (int i = i_first; i < B; i += i_step) {
         uint32_t key_q[NPL];
@@ -123,18 +131,22 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         for (int k = 0; k < K; ++k) sum += __shfl_sync(0xffffffffu, ex, k);  // slot order, like the definition
         if (lane < K) {
             const double wv = ex / sum;
-            sm0->ids[i * K + lane] = my_id;
-            sm0->w64[i * K + lane] = wv;
-            atomicAdd(&sm0->acc[my_id], (unsigned long long)(wv * 9007199254740992.0));  // 2^53
-            sm0->in_union[my_id] = 1;
+            // fixed-point (2^-53) integer atomics: the sum does not depend on the order of arrival
+            const unsigned long long fx = (unsigned long long)(wv * 9007199254740992.0);
+#pragma unroll
+            for (int r = 0; r < kDecCluster; ++r)
+                if (r < nct) {
+                    peer[r]->ids[i * K + lane] = my_id;
+                    peer[r]->w64[i * K + lane] = wv;
+                    atomicAdd(&peer[r]->acc[my_id], fx);
+                    peer[r]->in_union[my_id] = 1;
+                }
         }
     }
-    cluster.sync();  // every CTA's routes and sums have landed in the first CTA
-    if (rank != 0) return;
+    cluster.sync();  // all routes and sums have landed in every copy
     DEC_T(2);
 
     const int nslots = B * K;
-    const bool is_static = p.st_pool != nullptr;
     if (is_static) {
         // static pool: precomputed pool, targets and scalars; no batch reduction
         for (int e = threadIdx.x; e < N; e += kDecThreads) {
@@ -150,7 +162,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         }
         if (threadIdx.x == 0) sm.P = M;
     }
-    // ---- Eq. 11: score_e = h_e * sum_i w_{i,e}
+    // ---- Eq. 11: score_e = h_e * sum_i w_{i,e} (every CTA computes the same pool from the same sums)
     if (!is_static)
         for (int e = threadIdx.x; e < N; e += kDecThreads)
             sm.score[e] = (double)sm.acc[e] * (1.0 / 9007199254740992.0) * (double)p.h[e];
@@ -180,83 +192,70 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     __syncthreads();
     DEC_T(4);
     const int P = sm.P;
-    // ---- Eq. 12 for every source expert: itself if in the pool, else its min-loss pool expert.
-    // A warp takes up to 8 sources at a time and issues all their loss loads before reducing, then
-    // all their scalar loads: two rounds of memory latency per batch instead of two per source.
-    for (int s0 = warp * 8; s0 < N && !is_static; s0 += kWarps * 8) {
-        float bl[8];
-        int bt[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int s = s0 + u;
-            bl[u] = INFINITY;
-            bt[u] = 0x7fffffff;
-            if (s < N && sm.rank_of[s] < 0) {
+    // ---- Eq. 12 for the source experts of this CTA's slice (one warp per source, table rows in shared
+    // memory): itself if in the pool, else its min-loss pool expert; the result goes to every copy.
+    if (!is_static) {
+        for (int s = s_lo + warp; s < s_hi; s += kWarps) {
+            int bt = s;
+            float sc = 1.0f;
+            if (sm.rank_of[s] < 0) {  // warp-uniform
+                const float* row = tL + (size_t)(s - s_lo) * N;
+                float bl = INFINITY;
+                int bj = 0x7fffffff;
                 for (int j = lane; j < P; j += 32) {
                     const int t = sm.pool[j];
-                    const float l = __ldg(p.L + (size_t)s * N + t);
-                    if (bt[u] == 0x7fffffff || l < bl[u] || (l == bl[u] && t < bt[u])) {
-                        bl[u] = l;
-                        bt[u] = t;
+                    const float l = row[t];
+                    if (bj == 0x7fffffff || l < bl || (l == bl && t < bj)) {
+                        bl = l;
+                        bj = t;
                     }
                 }
+                bt = warp_argmin(bj != 0x7fffffff, float_order_key(bl), bj);
+                sc = tS[(size_t)(s - s_lo) * N + bt];
+            }
+            if (lane < nct) {
+                DecSmem* dst = cluster.map_shared_rank(&sm, lane);
+                dst->target[s] = bt;
+                dst->scale[s] = sc;
             }
         }
-        float sc[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int s = s0 + u;
-            sc[u] = 1.0f;
-            if (s < N) {  // warp-uniform
-                if (sm.rank_of[s] >= 0) bt[u] = s;
-                else {
-                    bt[u] = warp_argmin(bt[u] != 0x7fffffff, float_order_key(bl[u]), bt[u]);
-                    if (lane == 0) sc[u] = __ldg(p.S + (size_t)s * N + bt[u]);
-                }
-            }
-        }
-        if (lane == 0) {
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int s = s0 + u;
-                if (s < N) {
-                    sm.target[s] = bt[u];
-                    sm.scale[s] = sc[u];
-                }
-            }
-        }
+        cluster.sync();  // targets of all slices are in every copy
     }
-    __syncthreads();
     DEC_T(5);
-    // ---- Eq. 14: remap every slot in place; [B][K] layout kept
+    // ---- Eq. 14: remap every slot in place (each CTA on its own copy); [B][K] layout kept
     for (int s = threadIdx.x; s < nslots; s += kDecThreads) {
         int e = sm.ids[s];
         int t = sm.target[e];
         float wv = (float)(sm.w64[s] * (double)sm.scale[e]);
         sm.ids[s] = t;
         sm.wrm[s] = wv;
-        p.ids[s] = t;
-        p.w[s] = wv;
-    }
-    for (int e = threadIdx.x; e < N; e += kDecThreads) {
-        p.target[e] = sm.target[e];
-        p.scale[e] = sm.scale[e];
-        p.pool_ids[e] = e < P ? sm.pool[e] : -1;
-    }
-    if (threadIdx.x < 8) {
-        uint32_t m = 0;
-        for (int b = 0; b < 32; ++b) {
-            int e = threadIdx.x * 32 + b;
-            if (e < N && sm.rank_of[e] >= 0) m |= 1u << b;
+        if (rank == 0) {
+            p.ids[s] = t;
+            p.w[s] = wv;
         }
-        p.pool_mask[threadIdx.x] = m;
     }
-    if (threadIdx.x == 0) *p.pool_size = P;
+    if (rank == 0) {
+        for (int e = threadIdx.x; e < N; e += kDecThreads) {
+            p.target[e] = sm.target[e];
+            p.scale[e] = sm.scale[e];
+            p.pool_ids[e] = e < P ? sm.pool[e] : -1;
+        }
+        if (threadIdx.x < 8) {
+            uint32_t m = 0;
+            for (int b = 0; b < 32; ++b) {
+                int e = threadIdx.x * 32 + b;
+                if (e < N && sm.rank_of[e] >= 0) m |= 1u << b;
+            }
+            p.pool_mask[threadIdx.x] = m;
+        }
+        if (threadIdx.x == 0) *p.pool_size = P;
+    }
     __syncthreads();
     DEC_T(6);
-    // ---- execution lists: one row per distinct (token, pool expert), grouped by pool rank
+    // ---- execution lists: one row per distinct (token, pool expert), grouped by pool rank. Groups are
+    // dealt round-robin over the cluster's CTAs; pass 0 counts and broadcasts, pass 1 writes the rows.
     for (int pass = 0; pass < 2; ++pass) {
-        for (int g = warp; g < P; g += kWarps) {
+        for (int g = rank + nct * warp; g < P; g += nct * kWarps) {
             const int t = sm.pool[g];
             int run = pass ? sm.goff[g] : 0;
             for (int i0 = 0; i0 < B; i0 += 32) {
@@ -277,23 +276,34 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
                 }
                 run += __popc(m);
             }
-            if (!pass && lane == 0) sm.gcnt[g] = run;
+            if (!pass && lane < nct) cluster.map_shared_rank(&sm, lane)->gcnt[g] = run;
         }
-        __syncthreads();
         if (!pass) {
-            if (threadIdx.x == 0) {
-                int off = 0;
-                for (int g = 0; g < P; ++g) {
-                    sm.goff[g] = off;
-                    off += sm.gcnt[g];
+            cluster.sync();  // all group sizes are in every copy
+            if (warp == 0) {  // exclusive prefix over the groups, 32 at a time
+                int carry = 0;
+                for (int g0 = 0; g0 < P; g0 += 32) {
+                    const int g = g0 + lane;
+                    const int c = g < P ? sm.gcnt[g] : 0;
+                    int incl = c;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= o) incl += v;
+                    }
+                    if (g < P) sm.goff[g] = carry + incl - c;
+                    carry += __shfl_sync(0xffffffffu, incl, 31);
                 }
-                sm.goff[P] = off;
-                if (p.n_shared) sm.goff[P + 1] = off + B;
+                if (lane == 0) {
+                    sm.goff[P] = carry;
+                    if (p.n_shared) sm.goff[P + 1] = carry + B;
+                }
             }
             __syncthreads();
         }
     }
     DEC_T(7);
+    if (rank != 0) return;
     const int G = P + (p.n_shared ? 1 : 0);
     for (int g = threadIdx.x; g <= G; g += kDecThreads) {
         p.grp_off[g] = sm.goff[g];
@@ -318,6 +328,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     }
     DEC_T(8);
 }
+
 
 // Static pool: pool = TopK_e(h_e, M) (ties -> lower id, descending h), then Eq. 12 for every source.
 __global__ void __launch_bounds__(256) static_pool_kernel(int N, int M, const float* __restrict__ S,
@@ -393,7 +404,8 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const void* __restrict
 
 cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s) {
     const int npl = (p.N + 31) / 32;
-    const size_t smem = sizeof(DecSmem);
+    // state + this CTA's rows of the two tables
+    const size_t smem = kDecSmemBytes + 2 * (size_t)((p.N + kDecCluster - 1) / kDecCluster) * p.N * sizeof(float);
     cudaError_t err = cudaSuccess;
 #define EXFOLD_DEC_LAUNCH(NPL)                                                                              \
     err = cudaFuncSetAttribute(decode_route_kernel<NPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
