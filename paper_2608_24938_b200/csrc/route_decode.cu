@@ -38,11 +38,16 @@ struct DecSmem {
     int pool[kMaxExperts];      // pool ids by rank
     int target[kMaxExperts];
     float scale[kMaxExperts];
+    float hh[kMaxExperts];      // norm table h
     int gcnt[kMaxExperts + 2];
     int goff[kMaxExperts + 2];
     int P;
 };
 constexpr size_t kDecSmemBytes = (sizeof(DecSmem) + 15) / 16 * 16;  // the table rows follow
+
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(ptx::smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
 
 template <int NPL>
 __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRouteParams p) {
@@ -71,6 +76,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     for (int e = threadIdx.x; e < N; e += kDecThreads) {
         sm.acc[e] = 0ull;
         sm.in_union[e] = 0;
+        sm.rank_of[e] = -1;  // pool ranks arrive from other CTAs later
     }
     cluster.sync();  // every copy is cleared before any CTA adds to it
     // ---- Eq. 2 per token (warp per token, tokens dealt round-robin over the cluster's CTAs), weights in
@@ -82,14 +88,17 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         const int e = lane + 32 * q;
         vn[q] = (i_first < B && e < N) ? p.logits[(size_t)i_first * N + e] : -INFINITY;
     }
-    if (!is_static) {  // rows [s_lo, s_hi) of L and S: needed once the pool is known, in flight during the Top-K
+    if (!is_static) {
+        // Rows [s_lo, s_hi) of L and S and the norm table, needed once the sums are in: asynchronous copies
+        // into shared memory that stay in flight during the Top-K (waited for before the next cluster barrier).
         const int n_el = (s_hi - s_lo) * N;
         const float* gL = p.L + (size_t)s_lo * N;
         const float* gS = p.S + (size_t)s_lo * N;
         for (int idx = threadIdx.x; idx < n_el; idx += kDecThreads) {
-            tL[idx] = __ldg(gL + idx);
-            tS[idx] = __ldg(gS + idx);
+            cp_async4(tL + idx, gL + idx);
+            cp_async4(tS + idx, gS + idx);
         }
+        for (int e = threadIdx.x; e < N; e += kDecThreads) cp_async4(&sm.hh[e], p.h + e);
     }
     for (int i = i_first; i < B; i += i_step) {
         uint32_t key_q[NPL];
@@ -143,7 +152,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
                 }
         }
     }
-    cluster.sync();  // all routes and sums have landed in every copy
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    cluster.sync();  // all routes and sums have landed in every copy; this CTA's table rows are in place
     DEC_T(2);
 
     const int nslots = B * K;
@@ -165,31 +175,35 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     // ---- Eq. 11: score_e = h_e * sum_i w_{i,e} (every CTA computes the same pool from the same sums)
     if (!is_static)
         for (int e = threadIdx.x; e < N; e += kDecThreads)
-            sm.score[e] = (double)sm.acc[e] * (1.0 / 9007199254740992.0) * (double)p.h[e];
+            sm.score[e] = (double)sm.acc[e] * (1.0 / 9007199254740992.0) * (double)sm.hh[e];
     __syncthreads();
     DEC_T(3);
-    // pool = best min(M, |U|) experts of the union by (score desc, id asc): rank by counting,
-    // four threads per expert
+    // pool = best min(M, |U|) experts of the union by (score desc, id asc): rank by counting. Experts are
+    // dealt round-robin over the CTAs, one warp per expert; ranks are broadcast to every copy.
     if (!is_static) {
-        const int e = threadIdx.x >> 2, part = threadIdx.x & 3;  // 1024 threads cover 256 experts
-        const int in_u = (e < N) ? sm.in_union[e] : 0;
-        int better = 0;
-        if (in_u) {
+        int usz = 0;
+        for (int o = lane; o < N; o += 32) usz += sm.in_union[o] ? 1 : 0;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) usz += __shfl_xor_sync(0xffffffffu, usz, off);
+        if (threadIdx.x == 0) sm.P = usz < M ? usz : M;
+        for (int e = rank + nct * warp; e < N; e += nct * kWarps) {
+            if (!sm.in_union[e]) continue;  // warp-uniform
             const double se = sm.score[e];
-            for (int o = part; o < N; o += 4)
+            int better = 0;
+            for (int o = lane; o < N; o += 32)
                 if (sm.in_union[o] && (sm.score[o] > se || (sm.score[o] == se && o < e))) better++;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) better += __shfl_xor_sync(0xffffffffu, better, off);
+            if (better < M && lane < nct) {
+                DecSmem* dst = cluster.map_shared_rank(&sm, lane);
+                dst->rank_of[e] = better;
+                dst->pool[better] = e;
+            }
         }
-        better += __shfl_xor_sync(0xffffffffu, better, 1);
-        better += __shfl_xor_sync(0xffffffffu, better, 2);
-        const int usize = __syncthreads_count(in_u && part == 0);
-        if (e < N && part == 0) {
-            const int rk = (in_u && better < M) ? better : -1;
-            sm.rank_of[e] = rk;
-            if (rk >= 0) sm.pool[rk] = e;
-        }
-        if (threadIdx.x == 0) sm.P = usize < M ? usize : M;
+        cluster.sync();  // the pool is in every copy
+    } else {
+        __syncthreads();
     }
-    __syncthreads();
     DEC_T(4);
     const int P = sm.P;
     // ---- Eq. 12 for the source experts of this CTA's slice (one warp per source, table rows in shared
