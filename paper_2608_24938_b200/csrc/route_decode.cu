@@ -78,7 +78,10 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         sm.in_union[e] = 0;
         sm.rank_of[e] = -1;  // pool ranks arrive from other CTAs later
     }
-    cluster.sync();  // every copy is cleared before any CTA adds to it
+    // Every copy must be cleared before any CTA adds to it: arrive now, wait just before the first remote
+    // write, so the barrier's latency hides behind the logits load and the Top-K rounds.
+    cluster.barrier_arrive();
+    bool cleared = false;
     // ---- Eq. 2 per token (warp per token, tokens dealt round-robin over the cluster's CTAs), weights in
     // double; the first token's logits are requested before the table rows so that they arrive first.
     const int i_first = rank + nct * warp, i_step = nct * kWarps;
@@ -138,6 +141,10 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         double ex = lane < K ? exp((double)my_r - (double)rmax) : 0.0;
         double sum = 0.0;
         for (int k = 0; k < K; ++k) sum += __shfl_sync(0xffffffffu, ex, k);  // slot order, like the definition
+        if (!cleared) {  // warp-uniform
+            cluster.barrier_wait();
+            cleared = true;
+        }
         if (lane < K) {
             const double wv = ex / sum;
             // fixed-point (2^-53) integer atomics: the sum does not depend on the order of arrival
@@ -152,6 +159,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
                 }
         }
     }
+    if (!cleared) cluster.barrier_wait();  // warps without a token
     asm volatile("cp.async.wait_all;" ::: "memory");
     cluster.sync();  // all routes and sums have landed in every copy; this CTA's table rows are in place
     DEC_T(2);
