@@ -112,6 +112,22 @@ int orc_gate(const float *logits, int64_t T, int N, int K, int32_t *ids, float *
     return 0;
 }
 
+/* ---- router scores entering Eq. 2: r_e(x) = <W_r[e], x>, summed in double in index order;
+ *      out32 (fp32, what the layer consumes) and out64 may each be NULL ---- */
+int orc_router_logits(const void *x, int dtype, int64_t T, int d, const void *wr, int N, float *out32, double *out64)
+{
+    if (T < 0 || d < 1 || N < 1) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < T; ++i)
+        for (int e = 0; e < N; ++e) {
+            double r = 0.0;
+            for (int c = 0; c < d; ++c) r += ldv(wr, dtype, (size_t)e * d + c) * ldv(x, dtype, (size_t)i * d + c);
+            if (out32) out32[i * N + e] = (float)r;
+            if (out64) out64[i * N + e] = r;
+        }
+    return 0;
+}
+
 /* ---- Eq. 1: E_e(x) = W_down ( silu(W_gate x) * (W_up x) ) ---- */
 static void expert_ffn(const void *x, size_t xoff, int dtype, int d, int I,
                        const void *wg, const void *wu, const void *wd, int e,

@@ -70,6 +70,20 @@ def gate(logits: np.ndarray, K: int):
     return ids, w, w64
 
 
+def router_logits(x, wr):
+    """Router scores r = W_r x that Eq. 2 ranks. Returns (float32 [T,N], float64 [T,N])."""
+    x, wr = _c(x), _c(wr)
+    assert x.dtype == wr.dtype
+    T, d = x.shape
+    N = wr.shape[0]
+    assert wr.shape == (N, d)
+    r32 = np.empty((T, N), np.float32)
+    r64 = np.empty((T, N), np.float64)
+    rc = _L().orc_router_logits(_p(x), _dt(x), C.c_int64(T), d, _p(wr), N, _p(r32), _p(r64))
+    assert rc == 0, rc
+    return r32, r64
+
+
 def moe_apply(x, wg, wu, wd, ids, w, n_experts: int, n_shared: int = 0, tok_idx=None) -> np.ndarray:
     """y_i = sum_j w[i,j] E_{ids[i,j]}(x_i) (+ shared expert). Returns float32 [n_sel, d]."""
     x, wg, wu, wd = _c(x), _c(wg), _c(wu), _c(wd)

@@ -496,3 +496,28 @@ def test_oracle_regression_snapshot():
         else:
             np.testing.assert_allclose(np.asarray(now[k], np.float64), np.asarray(v, np.float64), rtol=1e-6, atol=1e-9,
                                        err_msg=k)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_router_logits_against_library_matmul_and_closed_forms(dtype):
+    """r = W_r x (the scores Eq. 2 ranks): equals a float64 library matmul of the same bit patterns; one-hot
+    router rows read single coordinates of x (a transposed operand or a wrong stride fails this); a constant
+    row e+1 against x = 1 gives d (e+1)."""
+    g = torch.Generator().manual_seed(7)
+    T, N, d = 13, 5, 24
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    x = torch.randn(T, d, generator=g).to(tdt)
+    wr = (0.3 * torch.randn(N, d, generator=g)).to(tdt)
+    r32, r64 = oracle.router_logits(A(x), A(wr))
+    ref = x.to(torch.float64) @ wr.to(torch.float64).T
+    np.testing.assert_allclose(r64, ref.numpy(), rtol=1e-13, atol=1e-13)
+    assert np.array_equal(r32, r64.astype(np.float32))
+    onehot = torch.zeros(N, d)
+    cols = [3, 0, 23, 7, 11]
+    for e, c in enumerate(cols):
+        onehot[e, c] = 1.0
+    r32, _ = oracle.router_logits(A(x), A(onehot.to(tdt)))
+    assert np.array_equal(r32, x.to(torch.float32).numpy()[:, cols])
+    const = (torch.arange(1, N + 1, dtype=torch.float32)[:, None] * torch.ones(N, d)).to(tdt)
+    r32, _ = oracle.router_logits(A(torch.ones(T, d).to(tdt)), A(const))
+    assert np.array_equal(r32, np.tile(d * np.arange(1, N + 1, dtype=np.float32), (T, 1)))
