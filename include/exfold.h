@@ -207,6 +207,18 @@ int exfold_moe_decode_static(const exfold_layer *layer, const void *x, const flo
                              void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Router scores that Eq. 2 ranks: logits[i][e] = <w_router[e], x[i]> for T tokens, fp32 out.
+ * x [T][d] and w_router [N][d] are in the layer dtype (device), logits [T][N] fp32 (device, 16-byte aligned).
+ * bf16 layers run on the tensor cores (bf16 products, fp32 accumulation, order unspecified); fp32 layers on
+ * an fp32 dot-product kernel. The result is the `logits` argument of the prefill / decode calls; a Top-K
+ * decision on scores closer than the accumulation error (~1e-6 relative) is not reproducible bit for bit
+ * against another summation order. Workspace: exfold_workspace_bytes(layer, T, 1). Enqueues on the stream
+ * and returns without synchronising. The shared expert and the tables play no part.
+ */
+int exfold_router_logits(const exfold_layer *layer, const void *x, const void *w_router, int64_t T, float *logits,
+                         void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * The same two calls for activations that live in HOST memory (pinned for real overlap):
  * x_host, logits_host and y_host are host pointers; the call stages them through the
  * workspace with asynchronous copies on the stream (x and logits in before the layer, y out

@@ -30,7 +30,7 @@ EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibr
            "exfold_moe_decode", "exfold_moe_prefill_host", "exfold_moe_decode_host", "exfold_device_status",
            "exfold_status_string", "exfold_launch_count", "exfold_profile_enable", "exfold_profile_read",
            "exfold_moe_decode_noalloc", "exfold_static_pool_build", "exfold_moe_decode_static",
-           "exfold_moe_prefill_ex"]
+           "exfold_moe_prefill_ex", "exfold_router_logits"]
 PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
                  "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
                  "simt_combine"]
@@ -95,6 +95,8 @@ def _load() -> C.CDLL:
     lib.exfold_moe_prefill_ex.restype = C.c_int
     lib.exfold_moe_prefill_ex.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables), i32,
                                           C.POINTER(exfold_fold_opts), vp, C.POINTER(exfold_prefill_meta), vp, sz, vp]
+    lib.exfold_router_logits.restype = C.c_int
+    lib.exfold_router_logits.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, sz, vp]
     lib.exfold_static_pool_build.restype = C.c_int
     lib.exfold_static_pool_build.argtypes = [C.POINTER(exfold_layer), C.POINTER(exfold_tables), i32,
                                              C.POINTER(exfold_static_pool), vp]
@@ -186,6 +188,11 @@ def alloc_workspace(layer: exfold_layer, max_tokens: int, routes_per_token: int,
     if host_staging:
         n += exfold_host_staging_bytes(layer, max_tokens)
     return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def exfold_router_logits(layer, x, w_router, logits, ws, stream=None) -> int:
+    return int(lib.exfold_router_logits(C.byref(layer), _ptr(x), _ptr(w_router), x.shape[0], _ptr(logits), _ptr(ws),
+                                        ws.numel(), _stream(stream)))
 
 
 def exfold_device_status(ws: torch.Tensor, stream=None) -> int:

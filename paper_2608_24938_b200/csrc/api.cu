@@ -622,6 +622,47 @@ int exfold_calibrate(const exfold_layer* layer, const void* x_cal, const float* 
     return un > 0 ? EXFOLD_WARN_UNOBSERVED_EXPERT : EXFOLD_OK;
 }
 
+int exfold_router_logits(const exfold_layer* layer, const void* x, const void* w_router, int64_t T, float* logits,
+                         void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (!valid_layer(layer) || !x || !w_router || !logits || !ws || T < 1) return EXFOLD_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ws) & 255) != 0 || (reinterpret_cast<uintptr_t>(logits) & 15) != 0)
+        return EXFOLD_ERR_INVALID_ARG;
+    const exfold_layer& l = *layer;
+    const int N = l.n_experts, d = l.hidden;
+    if (T > (int64_t)1 << 30) return EXFOLD_ERR_UNSUPPORTED;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
+    exfold_layer lc = l;
+    lc.n_shared = 0;
+    const Plan pl = make_plan(lc, T, 1);
+    if (ws_bytes < pl.total) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
+    EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
+    if (l.dtype == EXFOLD_F32) {
+        EXFOLD_CUDA(launch_router_simt(reinterpret_cast<const float*>(x), reinterpret_cast<const float*>(w_router), T, N,
+                                       d, logits, s));
+        return EXFOLD_OK;
+    }
+    // bf16: one group of T rows through GEMM-2's instantiation of the grouped kernel (K = d, N output columns in
+    // one 256-column tile, raw fp32 row epilogue); W_r rows past N are zero-filled by the tensor map
+    if (!aligned16(x) || !aligned16(w_router)) return EXFOLD_ERR_INVALID_ARG;
+    CUtensorMap tm_x, tm_wr;
+    if (!make_tmap(&tm_x, x, (uint64_t)T, d, 128) || !make_tmap(&tm_wr, w_router, (uint64_t)N, d, 256))
+        return EXFOLD_ERR_CUDA;
+    int32_t* offsets = at<int32_t>(ws, pl.offsets);
+    int32_t* work_start = at<int32_t>(ws, pl.work_start);
+    EXFOLD_CUDA(launch_calib_common_rows(offsets, work_start, T, 1, s));  // offsets {0, T}, tiles {0, ceil(T/128)}
+    GroupedGemmParams g{};
+    g.tm_a = tm_x; g.tm_a2 = tm_x; g.tm_b0 = tm_wr; g.tm_b1 = tm_wr;
+    g.offsets = offsets; g.work_start = work_start; g.G = 1; g.n_routed = 1; g.R = (int)T; g.x_rows = (int)T;
+    g.d = N;   // output width
+    g.I = d;   // contraction length
+    g.n_ntiles = 1; g.ksplit = 1; g.a_rows = kTileM;
+    g.row_tok = at<int32_t>(ws, pl.row_tok); g.row_w = at<float>(ws, pl.row_w);  // read, not used, by this epilogue
+    g.o32 = logits; g.status = at<DeviceStatus>(ws, pl.status);
+    const int64_t tiles = (T + kTileM - 1) / kTileM;
+    EXFOLD_CUDA(launch_grouped_gemm2(g, (int)std::min<int64_t>(sm_count(), tiles), s));
+    return EXFOLD_OK;
+}
+
 int exfold_moe_prefill_host(const exfold_layer* layer, const void* x_host, const float* logits_host, int64_t T,
                             const void* w_gate, const void* w_up, const void* w_down, const exfold_tables* tables,
                             int32_t k_pre, void* y_host, const exfold_prefill_meta* meta, void* ws, size_t ws_bytes,

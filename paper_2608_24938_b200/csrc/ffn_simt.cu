@@ -130,7 +130,32 @@ __global__ void convert_bf16_kernel(const float4* __restrict__ src, int64_t n4, 
     }
 }
 
+// r[i][e] = <W_r[e], x_i> in fp32, one warp per (token, expert): fp32 layers
+__global__ void __launch_bounds__(256) router_simt_kernel(const float* __restrict__ x, const float* __restrict__ wr,
+                                                          int64_t T, int N, int d, float* __restrict__ out) {
+    const int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (w >= T * N) return;
+    const int64_t i = w / N;
+    const int e = (int)(w % N);
+    const float* xi = x + i * d;
+    const float* we = wr + (size_t)e * d;
+    float acc = 0.f;
+    for (int c = lane; c < d; c += 32) acc = fmaf(we[c], xi[c], acc);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (lane == 0) out[w] = acc;
+}
+
 }  // namespace
+
+cudaError_t launch_router_simt(const float* x, const float* wr, int64_t T, int N, int d, float* out, cudaStream_t s) {
+    const int64_t warps = T * N;
+    if (warps == 0) return cudaSuccess;
+    router_simt_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, s>>>(x, wr, T, N, d, out);
+    count_launch();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_simt_ffn(const SimtFfnParams& p, cudaStream_t s) {
     const int64_t rows = p.T * p.Kr + p.T * p.n_shared;

@@ -289,12 +289,19 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                     ptx::tmem_ld_wait();
                     const int col0 = it.n_idx * 256 + c * 32;
                     if (valid && col0 < p.d) {
-                        if (!DEC && p.o32 != nullptr) {  // calibration: raw fp32 expert outputs by sorted row
-                            float4* dst = reinterpret_cast<float4*>(p.o32 + grow * p.d + col0);
+                        if (!DEC && p.o32 != nullptr) {  // raw fp32 rows (calibration outputs, router scores)
+                            float* dstf = p.o32 + grow * p.d + col0;
+                            if (col0 + 32 <= p.d && (p.d & 3) == 0) {
+                                float4* dst = reinterpret_cast<float4*>(dstf);
 #pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                                for (int j = 0; j < 8; ++j)
+                                    dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                         __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                            } else {  // ragged or unaligned row end
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (col0 + j < p.d) dstf[j] = __uint_as_float(v[j]);
+                            }
                         } else if (p.y32 != nullptr) {
                             float* dst = p.y32 + (int64_t)tok * p.d + col0;
 #pragma unroll

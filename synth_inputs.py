@@ -24,7 +24,7 @@ import torch
 # tensor tags for the sub-streams
 _TAG = {"x": 1, "logits": 2, "w_gate": 3, "w_up": 4, "w_down": 5, "tables": 6,
         "x_cal": 7, "logits_cal": 8, "zipf_perm": 9, "x_dec": 10, "logits_dec": 11,
-        "corr_base": 12, "corr_gain": 13}
+        "corr_base": 12, "corr_gain": 13, "w_router": 14}
 
 
 @dataclasses.dataclass(frozen=True)
@@ -107,6 +107,13 @@ def router_logits(cfg: LayerConfig, n_tokens: int, tag: str = "logits") -> torch
 
 def _one_expert(cfg: LayerConfig, tag: str, e: int, shape, std: float) -> torch.Tensor:
     return to_dtype(_normal(cfg.seed, tag, e, shape, std), cfg.dtype)
+
+
+def router_weights(cfg: LayerConfig, std: Optional[float] = None) -> torch.Tensor:
+    """Router matrix W_r [N, d] in the layer dtype, entries N(0, std); the default std = 1/sqrt(d) gives
+    unit-variance scores on x ~ N(0, 1), like the logits generator's "normal" mode."""
+    std = (1.0 / np.sqrt(cfg.hidden)) if std is None else std
+    return to_dtype(_normal(cfg.seed, "w_router", 0, (cfg.n_experts, cfg.hidden), std), cfg.dtype)
 
 
 def expert_weights(cfg: LayerConfig, std: float = 0.02, threads: Optional[int] = None,

@@ -354,3 +354,60 @@ def test_host_buffer_entry_points():
     ex.exfold_moe_decode_host(case.layer, xdh, ldh, case.d_wg, case.d_wu, case.d_wd, case.tables, 6, ydh, ws)
     assert ex.exfold_device_status(ws) == 0
     check_output(ydh.float().numpy(), case.oracle_decode(6)["y"], "bf16")
+
+
+# ------------------------------------------------------------------ router scores (input of Eq. 2)
+@pytest.mark.parametrize("dtype,N,T", [("bf16", 16, 300), ("bf16", 8, 129), ("bf16", 200, 1000), ("bf16", 6, 77),
+                                       ("f32", 8, 64)])
+def test_router_logits_match_oracle(dtype, N, T):
+    """logits = x W_r^T on the tensor cores (bf16) / fp32 dot products: within 1e-4 of the largest score.
+    N = 8 and 6 end inside the first 32-column chunk (6: rows not 16-byte aligned), N = 200 spans seven."""
+    cfg = small_bf16(n_experts=N, top_k=2, dtype=dtype, prefill_tokens=T, hidden=256 if dtype == "bf16" else 128)
+    ex = Case(cfg).ex
+    dev = torch.device("cuda:0")
+    x, wr = si.hidden_states(cfg, T), si.router_weights(cfg)
+    ref32, _ = oracle.router_logits(A(x), A(wr))
+    layer = ex.make_layer(N, 0, cfg.hidden, cfg.inter, cfg.top_k, cfg.dtype)
+    ws = ex.alloc_workspace(layer, T, 1)
+    ws.fill_(0xFF)
+    lg = torch.full((T, N), float("nan"), device=dev)
+    assert ex.exfold_router_logits(layer, x.to(dev), wr.to(dev), lg, ws) == 0
+    assert ex.exfold_device_status(ws) == 0
+    got = lg.cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref32).max() <= 1e-4 * np.abs(ref32).max()
+
+
+def test_router_then_prefill_chain():
+    """Scores from the GPU router feed the folded prefill; the oracle runs its own scores through its own layer.
+    Tokens whose ranking-relevant gaps (between the Top-(K+1) scores, and between retained-set keys) exceed the
+    accumulation error must agree bit for bit in routing; the outputs of those tokens agree to the bf16 bound."""
+    cfg = small_bf16(n_experts=16, top_k=4, prefill_tokens=400)
+    case = Case(cfg)
+    ex, dev = case.ex, case.dev
+    T, N, K, Kp = 400, 16, 4, 2
+    wr = si.router_weights(cfg)
+    ref32, ref64 = oracle.router_logits(A(case.x), A(wr))
+    ws = ex.alloc_workspace(case.layer, T, K)
+    lg = torch.empty((T, N), device=dev)
+    assert ex.exfold_router_logits(case.layer, case.d_x, wr.to(dev), lg, ws) == 0
+    got_lg = lg.cpu().numpy()
+    tol = 1e-4 * np.abs(ref32).max()
+    assert np.abs(got_lg - ref32).max() <= tol
+    # tokens that are safe against a perturbation of every score by tol
+    lnh = case.tables_host[3].numpy()
+    srt = np.sort(ref64, axis=1)[:, ::-1]
+    gap_topk = (srt[:, :K] - srt[:, 1:K + 1]).min(axis=1)
+    ids_ref, _, _ = oracle.gate(ref32, K)
+    keys = np.take_along_axis(ref64, ids_ref.astype(np.int64), 1) + lnh[ids_ref]
+    ks = np.sort(keys, axis=1)[:, ::-1]
+    gap_keys = (ks[:, :-1] - ks[:, 1:]).min(axis=1)
+    safe = (gap_topk > 4 * tol) & (gap_keys > 4 * tol)
+    assert safe.mean() > 0.9
+    case.lg, case.d_lg = torch.from_numpy(ref32), lg      # oracle side: its own scores; GPU side: the GPU's
+    ref = case.oracle_prefill(Kp)
+    got = case.run_prefill(Kp)
+    assert np.array_equal(got["ids"][safe], ref["ids"][safe])
+    assert np.array_equal(got["omit_tgt"][safe], ref["omit_tgt"][safe])
+    np.testing.assert_allclose(got["w"][safe], ref["w"][safe], rtol=2e-3, atol=1e-5)
+    check_output(got["y"][safe], ref["y"][safe], "bf16")
