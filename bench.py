@@ -171,6 +171,56 @@ def workload_config(args):
     return cfg
 
 
+def stack_leg(ex, cfg, layer, tables, weights, xd, M, L, dev, flush, reps=10):
+    """L decode layers of the workload's shape, each = router scores (W_r x) + folded decode layer, one after the
+    other on one stream. Every layer owns its weights (device copies rolled along the expert axis, so no weight
+    line is reused between layers) and its router matrix; all layers read the same x (the layers are sequential
+    in time, independent in data). Timed as plain stream launches and as one captured CUDA graph."""
+    import torch
+    wg, wu, wd = weights
+    B, N, d = xd.shape[0], cfg.n_experts, cfg.hidden
+    per = [(torch.roll(wg, l, 0), torch.roll(wu, l, 0), torch.roll(wd, l, 0)) if l else (wg, wu, wd) for l in range(L)]
+    wr0 = si.router_weights(cfg).to(dev)
+    wrs = [torch.roll(wr0, l, 0) for l in range(L)]
+    lgs = [torch.empty((B, N), dtype=torch.float32, device=dev) for _ in range(L)]
+    ys = [torch.empty((B, d), dtype=wg.dtype, device=dev) for _ in range(L)]
+    ws = ex.alloc_workspace(layer, B, cfg.top_k)
+
+    def run_layers():
+        for l in range(L):
+            ex.exfold_router_logits(layer, xd, wrs[l], lgs[l], ws)
+            ex.exfold_moe_decode(layer, xd, lgs[l], per[l][0], per[l][1], per[l][2], tables, M, ys[l], ws)
+
+    def timed(fn):
+        ts = []
+        for it in range(reps + 2):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    res = {"layers": L, "what": "router GEMM + folded decode layer per layer, own weights per layer, same x"}
+    res["stream_us_per_layer"] = timed(run_layers) * 1e3 / L
+    assert ex.exfold_device_status(ws) == 0, "device status after the layer stack"
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            run_layers()
+        torch.cuda.synchronize()
+        res["graph_us_per_layer"] = timed(graph.replay) * 1e3 / L
+        assert ex.exfold_device_status(ws) == 0, "device status after the graph replays"
+    except Exception as e:  # capture is an optional measurement: report, do not lose the benchmark line
+        res["graph_error"] = f"{type(e).__name__}: {e}"[:300]
+    return res
+
+
 def run_ours(args, rank, world):
     import torch
     import torch.distributed as dist
@@ -299,6 +349,11 @@ def run_ours(args, rank, world):
     h2d = T * d * el + T * N * 4 + B * d * el + B * N * 4
     d2h = T * d * el + B * d * el
 
+    # ---- optional: a stack of decode layers (router GEMM + folded decode layer), stream launches vs one CUDA graph
+    stack = None
+    if args.layers > 0 and world == 1:
+        stack = stack_leg(ex, cfg, layer, tables, (wg, wu, wd), xd, M, args.layers, dev, flush)
+
     # ---- algorithmic work
     rows = T * Kp + T * cfg.n_shared
     flop_layer = rows * 6.0 * d * I
@@ -332,6 +387,8 @@ def run_ours(args, rank, world):
         "peaks": {"source": peak_src, **peaks},
         "wall_s_timed_region": wall,
     }
+    if stack is not None:
+        out["stack"] = stack
     if "gemm1_gateup_swiglu" in kern:
         t1 = kern["gemm1_gateup_swiglu"] * 1e-3
         ach = flop_gemm1 / t1 / 1e12
@@ -435,6 +492,9 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="override the prefill token count (reduced cases for profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the decode batch")
     ap.add_argument("--inter", type=int, default=0, help="override the expert intermediate size")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="also time a stack of this many decode layers (router scores + folded decode layer each), "
+                         "launched on the stream and replayed as one CUDA graph")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-flop-budget", type=float, default=3e11,
                     help="flop of oracle work in the cpu-baseline sample (about 10-30 s of CPU time)")

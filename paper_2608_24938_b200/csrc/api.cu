@@ -647,12 +647,10 @@ int exfold_router_logits(const exfold_layer* layer, const void* x, const void* w
     CUtensorMap tm_x, tm_wr;
     if (!make_tmap(&tm_x, x, (uint64_t)T, d, 128) || !make_tmap(&tm_wr, w_router, (uint64_t)N, d, 256))
         return EXFOLD_ERR_CUDA;
-    int32_t* offsets = at<int32_t>(ws, pl.offsets);
-    int32_t* work_start = at<int32_t>(ws, pl.work_start);
-    EXFOLD_CUDA(launch_calib_common_rows(offsets, work_start, T, 1, s));  // offsets {0, T}, tiles {0, ceil(T/128)}
     GroupedGemmParams g{};
     g.tm_a = tm_x; g.tm_a2 = tm_x; g.tm_b0 = tm_wr; g.tm_b1 = tm_wr;
-    g.offsets = offsets; g.work_start = work_start; g.G = 1; g.n_routed = 1; g.R = (int)T; g.x_rows = (int)T;
+    g.offsets = nullptr; g.work_start = nullptr; g.G = 1;  // one group of R = T rows
+    g.n_routed = 1; g.R = (int)T; g.x_rows = (int)T;
     g.d = N;   // output width
     g.I = d;   // contraction length
     g.n_ntiles = 1; g.ksplit = 1; g.a_rows = kTileM;

@@ -121,8 +121,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         G = gd < G ? gd : G;
     }
     for (int i = threadIdx.x; i <= G; i += kGemmThreads) {
-        s_off[i] = p.offsets[i];
-        s_ws[i] = p.work_start[i];
+        // offsets == null: one group of p.R rows (a plain GEMM, e.g. the router scores)
+        s_off[i] = p.offsets != nullptr ? p.offsets[i] : i * p.R;
+        s_ws[i] = p.offsets != nullptr ? p.work_start[i] : i * ((p.R + kTileM - 1) / kTileM);
         if (DEC) s_exp[i] = i < G ? p.grp_expert[i] : i;  // group -> expert whose weights it uses
     }
     ptx::tc_fence_before();
