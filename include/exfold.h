@@ -224,6 +224,10 @@ int exfold_router_logits(const exfold_layer *layer, const void *x, const void *w
  * workspace with asynchronous copies on the stream (x and logits in before the layer, y out
  * after it). Weights, tables, metadata and workspace stay device pointers. The workspace
  * must be exfold_workspace_bytes(...) + exfold_host_staging_bytes(...) large.
+ * A prefill call of 4096 tokens or more that asks for no metadata is run as up to four chunks of whole
+ * 128-row tiles: the next chunk is copied in and the previous one copied out on two helper streams
+ * created and destroyed inside the call, while the caller's stream computes; the call still completes in
+ * the caller's stream order and the result is the same bit for bit (tokens do not interact).
  */
 size_t exfold_host_staging_bytes(const exfold_layer *layer, int64_t max_tokens);
 int exfold_moe_prefill_host(const exfold_layer *layer, const void *x_host, const float *logits_host,

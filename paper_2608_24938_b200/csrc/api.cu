@@ -24,6 +24,7 @@ namespace exfold {
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 static thread_local bool t_pdl = false;
+static thread_local bool t_keep_status = false;  // set while a host-buffer call runs its second and later chunks
 void set_pdl(bool on) { t_pdl = on; }
 bool pdl_enabled() { return t_pdl; }
 
@@ -152,6 +153,8 @@ EncodeTiledFn encode_fn() {
     }
     return fn;
 }
+
+constexpr int kMaxHostChunks = 4;  // host-buffer prefill: chunks of >= 2048 tokens in flight
 
 // bf16 matrix [rows][cols] row-major; box = box_rows x 64 columns (128 bytes), 128-byte swizzle
 bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
@@ -325,7 +328,8 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     rp.ids = at<int32_t>(ws, pl.ids); rp.w = at<float>(ws, pl.w);
     rp.omit_src = at<int32_t>(ws, pl.omit_src); rp.omit_tgt = at<int32_t>(ws, pl.omit_tgt);
     rp.block_hist = at<int32_t>(ws, pl.block_hist);
-    rp.status = at<DeviceStatus>(ws, pl.status);  // the first kernel of the call clears the status record
+    // the first kernel of the call clears the status record (not for the later chunks of a chunked host call)
+    rp.status = t_keep_status ? nullptr : at<DeviceStatus>(ws, pl.status);
     { ProfScope ps(0, s); EXFOLD_CUDA(launch_prefill_route(rp, s)); }
 
     PrefillScatterParams cp{};
@@ -676,12 +680,73 @@ int exfold_moe_prefill_host(const exfold_layer* layer, const void* x_host, const
     char* yd = xd + align_up(xb, 256);
     char* ld = yd + align_up(xb, 256);
     cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
-    EXFOLD_CUDA(cudaMemcpyAsync(xd, x_host, xb, cudaMemcpyHostToDevice, s));
-    EXFOLD_CUDA(cudaMemcpyAsync(ld, logits_host, lb, cudaMemcpyHostToDevice, s));
-    int rc = exfold_moe_prefill(layer, xd, reinterpret_cast<const float*>(ld), T, w_gate, w_up, w_down, tables, k_pre,
-                                yd, meta, ws, main_bytes, cuda_stream);
-    if (rc != EXFOLD_OK) return rc;
-    EXFOLD_CUDA(cudaMemcpyAsync(y_host, yd, xb, cudaMemcpyDeviceToHost, s));
+    // Tokens are independent, so a long prompt goes through in chunks: chunk c+1 is copied in and chunk c-1 copied
+    // out (two helper streams, both PCIe directions) while chunk c is computed on the caller's stream. Routing
+    // metadata describes the whole call (one permutation over all routes), so a call that asks for it is not split.
+    const int64_t chunk_tokens = 2048;
+    int chunks = meta != nullptr ? 1 : (int)std::min<int64_t>(kMaxHostChunks, T / chunk_tokens);
+    if (chunks <= 1) {
+        EXFOLD_CUDA(cudaMemcpyAsync(xd, x_host, xb, cudaMemcpyHostToDevice, s));
+        EXFOLD_CUDA(cudaMemcpyAsync(ld, logits_host, lb, cudaMemcpyHostToDevice, s));
+        int rc = exfold_moe_prefill(layer, xd, reinterpret_cast<const float*>(ld), T, w_gate, w_up, w_down, tables,
+                                    k_pre, yd, meta, ws, main_bytes, cuda_stream);
+        if (rc != EXFOLD_OK) return rc;
+        EXFOLD_CUDA(cudaMemcpyAsync(y_host, yd, xb, cudaMemcpyDeviceToHost, s));
+        return EXFOLD_OK;
+    }
+    struct Helpers {  // per-call helper streams and events; destruction is deferred by the runtime until they drain
+        cudaStream_t in = nullptr, out = nullptr;
+        cudaEvent_t start = nullptr, copied[kMaxHostChunks] = {}, computed[kMaxHostChunks] = {}, done = nullptr;
+        ~Helpers() {
+            if (start) cudaEventDestroy(start);
+            if (done) cudaEventDestroy(done);
+            for (int c = 0; c < kMaxHostChunks; ++c) {
+                if (copied[c]) cudaEventDestroy(copied[c]);
+                if (computed[c]) cudaEventDestroy(computed[c]);
+            }
+            if (in) cudaStreamDestroy(in);
+            if (out) cudaStreamDestroy(out);
+        }
+    } h;
+    EXFOLD_CUDA(cudaStreamCreateWithFlags(&h.in, cudaStreamNonBlocking));
+    EXFOLD_CUDA(cudaStreamCreateWithFlags(&h.out, cudaStreamNonBlocking));
+    EXFOLD_CUDA(cudaEventCreateWithFlags(&h.start, cudaEventDisableTiming));
+    EXFOLD_CUDA(cudaEventCreateWithFlags(&h.done, cudaEventDisableTiming));
+    for (int c = 0; c < chunks; ++c) {
+        EXFOLD_CUDA(cudaEventCreateWithFlags(&h.copied[c], cudaEventDisableTiming));
+        EXFOLD_CUDA(cudaEventCreateWithFlags(&h.computed[c], cudaEventDisableTiming));
+    }
+    // the staging buffers may still be in use by earlier work on the caller's stream
+    EXFOLD_CUDA(cudaEventRecord(h.start, s));
+    EXFOLD_CUDA(cudaStreamWaitEvent(h.in, h.start, 0));
+    EXFOLD_CUDA(cudaStreamWaitEvent(h.out, h.start, 0));
+    const size_t row_x = (size_t)layer->hidden * el, row_l = (size_t)layer->n_experts * 4;
+    const int64_t per = (T / chunks + 127) / 128 * 128;  // whole row tiles per chunk
+    for (int c = 0; c < chunks; ++c) {
+        const int64_t t0 = c * per, n = std::min<int64_t>(per, T - t0);
+        if (n <= 0) break;
+        EXFOLD_CUDA(cudaMemcpyAsync(xd + t0 * row_x, reinterpret_cast<const char*>(x_host) + t0 * row_x, n * row_x,
+                                    cudaMemcpyHostToDevice, h.in));
+        EXFOLD_CUDA(cudaMemcpyAsync(ld + t0 * row_l, reinterpret_cast<const char*>(logits_host) + t0 * row_l,
+                                    n * row_l, cudaMemcpyHostToDevice, h.in));
+        EXFOLD_CUDA(cudaEventRecord(h.copied[c], h.in));
+    }
+    for (int c = 0; c < chunks; ++c) {
+        const int64_t t0 = c * per, n = std::min<int64_t>(per, T - t0);
+        if (n <= 0) break;
+        EXFOLD_CUDA(cudaStreamWaitEvent(s, h.copied[c], 0));
+        t_keep_status = c > 0;  // an error recorded by an earlier chunk stays visible
+        int rc = exfold_moe_prefill(layer, xd + t0 * row_x, reinterpret_cast<const float*>(ld + t0 * row_l), n, w_gate,
+                                    w_up, w_down, tables, k_pre, yd + t0 * row_x, nullptr, ws, main_bytes, cuda_stream);
+        t_keep_status = false;
+        if (rc != EXFOLD_OK) return rc;
+        EXFOLD_CUDA(cudaEventRecord(h.computed[c], s));
+        EXFOLD_CUDA(cudaStreamWaitEvent(h.out, h.computed[c], 0));
+        EXFOLD_CUDA(cudaMemcpyAsync(reinterpret_cast<char*>(y_host) + t0 * row_x, yd + t0 * row_x, n * row_x,
+                                    cudaMemcpyDeviceToHost, h.out));
+    }
+    EXFOLD_CUDA(cudaEventRecord(h.done, h.out));
+    EXFOLD_CUDA(cudaStreamWaitEvent(s, h.done, 0));  // the call is complete, in the caller's stream order, when y_host is
     return EXFOLD_OK;
 }
 
