@@ -84,6 +84,16 @@ def test_bad_arguments_are_rejected_before_launch(ex):
     assert rc == ex.EXFOLD_ERR_INVALID_ARG                     # unknown calibration mode
     assert ex.lib.exfold_device_status(None, None) == ex.EXFOLD_ERR_INVALID_ARG
 
+    def router(layer=layer, x=p, wr=p, T=4, lg=p, ws=p, wsb=big):
+        return ex.lib.exfold_router_logits(C.byref(layer), x, wr, T, lg, ws, wsb, None)
+
+    assert router(x=None) == ex.EXFOLD_ERR_INVALID_ARG
+    assert router(wr=None) == ex.EXFOLD_ERR_INVALID_ARG
+    assert router(T=0) == ex.EXFOLD_ERR_INVALID_ARG
+    assert router(lg=p + 4) == ex.EXFOLD_ERR_INVALID_ARG       # logits not 16-byte aligned
+    assert router(ws=p + 8) == ex.EXFOLD_ERR_INVALID_ARG
+    assert router(wsb=64) == ex.EXFOLD_ERR_WORKSPACE_TOO_SMALL
+
 
 def test_product_package_does_not_touch_the_oracle():
     """The CUDA path and the oracle share no code and neither imports the other."""
