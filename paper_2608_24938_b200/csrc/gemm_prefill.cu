@@ -17,10 +17,15 @@
 #include "common.cuh"
 #include "ptx.cuh"
 
+#ifndef EXFOLD_TRACE_KB_MODE
+#define EXFOLD_TRACE_KB_MODE 0  // trace builds: which prefill GEMM (0 or 1) logs per-k-block timestamps
+#endif
+
 namespace exfold {
 
 namespace {
 
+constexpr int kTraceKb = 1280;  // trace builds: k-blocks logged (table 3 of the trace array holds 2 x 1280 words)
 constexpr int kBK = 64;                       // K elements per stage: 128 bytes = one swizzle row
 constexpr int kStages = 4;
 constexpr int kMaxStages = 6;  // decode loads a shorter A box per stage and fits more stages
@@ -193,6 +198,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         if (lane == 0) {
             constexpr uint32_t idesc = ptx::make_idesc_bf16(128, 256);
             int stage = 0, phase = 0, iter = 0;
+#ifdef EXFOLD_TRACE
+            int kbt = 0;
+#endif
             bool ok = true;
             for (int w = w_begin; w < total && ok; w += w_stride, ++iter) {
                 const int as = iter & 1, aphase = (iter >> 1) & 1;
@@ -211,6 +219,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                         break;
                     }
                     ptx::tc_fence_after();
+#ifdef EXFOLD_TRACE
+                    // one CTA of the chosen prefill GEMM logs when each k-block's operands were ready (cycles, ns)
+                    if (MODE == EXFOLD_TRACE_KB_MODE && !DEC && blockIdx.x == 5 && kbt < kTraceKb) {
+                        unsigned long long* flat = &g_trace[3][0][0];
+                        flat[kbt] = (unsigned long long)clock64();
+                        flat[kTraceKb + kbt] = ptx::globaltimer_ns();
+                        ++kbt;
+                    }
+#endif
                     const uint32_t a_addr = ptx::smem_u32(tiles + stage * stage_bytes);
                     const uint64_t adesc = ptx::make_kmajor_sw128_desc(a_addr);
                     const uint64_t bdesc = ptx::make_kmajor_sw128_desc(a_addr + a_bytes);
