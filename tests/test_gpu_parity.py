@@ -429,3 +429,38 @@ def test_host_prefill_in_chunks_equals_the_device_call():
         assert ex.exfold_device_status(ws) == 0
         assert np.array_equal(yh.float().numpy(), ref_dev)
     check_output(ref_dev[:256], case.oracle_prefill(1, tok_idx=np.arange(256))["y"], "bf16")
+
+
+# ------------------------------------------------------------------ seeded random shapes
+def _random_cfg(i):
+    """Shape i of a fixed, seeded family: odd expert counts, ragged token counts, every K' and M regime."""
+    rng = np.random.default_rng(1000 + i)
+    dtype = "bf16" if i % 4 != 3 else "f32"
+    N = int(rng.choice([3, 5, 8, 12, 24, 40, 64, 100]))
+    K = int(rng.integers(1, min(N, 9) + 1))
+    hidden = int(rng.choice([64, 128, 192, 320])) if dtype == "bf16" else int(rng.choice([32, 60, 100]))
+    inter = int(rng.choice([64, 128, 448])) if dtype == "bf16" else int(rng.choice([24, 50]))
+    T = int(rng.integers(1, 700))
+    B = int(rng.integers(1, 257)) if N * 1 else 1
+    while B * K > 4096:
+        B //= 2
+    return si.LayerConfig(f"rand{i}", N, int(rng.integers(0, 2)), hidden, inter, K, dtype, T, (1,), B, (1,),
+                          logits="zipf" if rng.random() < 0.5 else "normal", zipf_s=float(rng.choice([0.8, 1.1, 2.0])),
+                          seed=20260824 + i)
+
+
+@pytest.mark.parametrize("i", range(12))
+def test_random_shapes(i):
+    cfg = _random_cfg(i)
+    rng = np.random.default_rng(2000 + i)
+    case = Case(cfg, correlated=0.8 if i % 3 == 0 else 0.0)
+    Kp = int(rng.integers(1, cfg.top_k + 1))
+    got, ref = case.run_prefill(Kp), case.oracle_prefill(Kp)
+    assert ref["mismatch"] == 0  # the fp32 key and the fp64 product rank alike on these seeds
+    check_prefill_meta(got, ref)
+    check_output(got["y"], ref["y"], cfg.dtype)
+    M = int(rng.integers(1, cfg.n_experts + 1))
+    got, ref = case.run_decode(M), case.oracle_decode(M)
+    assert ref["min_gap"] > 1e-9   # no tie at the pool boundary on these seeds
+    check_decode_meta(got, ref, M)
+    check_output(got["y"], ref["y"], cfg.dtype)
