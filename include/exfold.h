@@ -209,8 +209,9 @@ int exfold_moe_decode_static(const exfold_layer *layer, const void *x, const flo
 /*
  * Router scores that Eq. 2 ranks: logits[i][e] = <w_router[e], x[i]> for T tokens, fp32 out.
  * x [T][d] and w_router [N][d] are in the layer dtype (device), logits [T][N] fp32 (device, 16-byte aligned).
- * bf16 layers run on the tensor cores (bf16 products, fp32 accumulation, order unspecified); fp32 layers on
- * an fp32 dot-product kernel. The result is the `logits` argument of the prefill / decode calls; a Top-K
+ * bf16 layers with more than 128 tokens run on the tensor cores (bf16 products, fp32 accumulation, order
+ * unspecified); fp32 layers and batches of at most 128 tokens on a dot-product kernel (fp32 accumulation in a
+ * fixed order). The result is the `logits` argument of the prefill / decode calls; a Top-K
  * decision on scores closer than the accumulation error (~1e-6 relative) is not reproducible bit for bit
  * against another summation order. Workspace: exfold_workspace_bytes(layer, T, 1). Enqueues on the stream
  * and returns without synchronising. The shared expert and the tables play no part.

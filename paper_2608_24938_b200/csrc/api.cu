@@ -640,9 +640,10 @@ int exfold_router_logits(const exfold_layer* layer, const void* x, const void* w
     const Plan pl = make_plan(lc, T, 1);
     if (ws_bytes < pl.total) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
     EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
-    if (l.dtype == EXFOLD_F32) {
-        EXFOLD_CUDA(launch_router_simt(reinterpret_cast<const float*>(x), reinterpret_cast<const float*>(w_router), T, N,
-                                       d, logits, s));
+    // fp32 layers, and bf16 batches of at most one row tile (decode): dot products in a fixed order. One 128-row
+    // tile on the tensor cores would walk the whole K loop on a single SM (10-19 us of latency).
+    if (l.dtype == EXFOLD_F32 || (T <= kTileM && aligned16(x) && aligned16(w_router))) {
+        EXFOLD_CUDA(launch_router_simt(x, w_router, l.dtype, T, N, d, logits, s));
         return EXFOLD_OK;
     }
     // bf16: one group of T rows through GEMM-2's instantiation of the grouped kernel (K = d, N output columns in

@@ -207,7 +207,8 @@ cudaError_t launch_simt_ffn(const SimtFfnParams& p, cudaStream_t s);
 // y[i] = sum_j w[i][j] out[i*Kr+j] (+ out[T*Kr+i] for the shared expert); y in the layer dtype
 cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, int Kr, int d, int n_shared,
                                   void* y, int dtype, cudaStream_t s);
-cudaError_t launch_router_simt(const float* x, const float* wr, int64_t T, int N, int d, float* out, cudaStream_t s);
+cudaError_t launch_router_simt(const void* x, const void* wr, int dtype, int64_t T, int N, int d, float* out,
+                               cudaStream_t s);
 cudaError_t launch_convert_bf16(const float* y32, int64_t n, void* y, cudaStream_t s);
 // y[i] = sum_j O[inv_pos[i*Kr+j]] (+ O[R+i] for the shared expert), fp32 sum in slot order, bf16 out
 cudaError_t launch_combine_rows(const __nv_bfloat16* O, const int32_t* inv_pos, int64_t T, int Kr, int d,

@@ -130,18 +130,34 @@ __global__ void convert_bf16_kernel(const float4* __restrict__ src, int64_t n4, 
     }
 }
 
-// r[i][e] = <W_r[e], x_i> in fp32, one warp per (token, expert): fp32 layers
-__global__ void __launch_bounds__(256) router_simt_kernel(const float* __restrict__ x, const float* __restrict__ wr,
-                                                          int64_t T, int N, int d, float* __restrict__ out) {
+// r[i][e] = <W_r[e], x_i>, fp32 accumulation in a fixed order, one warp per (token, expert): fp32 layers, and
+// bf16 batches too small to fill the tensor-core kernel (a single 128-row tile would walk K on one SM)
+template <typename T>
+__global__ void __launch_bounds__(256) router_simt_kernel(const T* __restrict__ x, const T* __restrict__ wr, int64_t Tn,
+                                                          int N, int d, float* __restrict__ out) {
     const int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
-    if (w >= T * N) return;
+    if (w >= Tn * N) return;
     const int64_t i = w / N;
     const int e = (int)(w % N);
-    const float* xi = x + i * d;
-    const float* we = wr + (size_t)e * d;
+    const T* xi = x + i * d;
+    const T* we = wr + (size_t)e * d;
     float acc = 0.f;
-    for (int c = lane; c < d; c += 32) acc = fmaf(we[c], xi[c], acc);
+    if constexpr (sizeof(T) == 2) {  // bf16: 8 elements (16 bytes) per lane and step; d is a multiple of 64
+        for (int c = lane * 8; c < d; c += 256) {
+            const uint4 a = *reinterpret_cast<const uint4*>(we + c), b = *reinterpret_cast<const uint4*>(xi + c);
+            const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+            const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 fa = __bfloat1622float2(pa[j]), fb = __bfloat1622float2(pb[j]);
+                acc = fmaf(fa.x, fb.x, acc);
+                acc = fmaf(fa.y, fb.y, acc);
+            }
+        }
+    } else {
+        for (int c = lane; c < d; c += 32) acc = fmaf((float)we[c], (float)xi[c], acc);
+    }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if (lane == 0) out[w] = acc;
@@ -149,10 +165,17 @@ __global__ void __launch_bounds__(256) router_simt_kernel(const float* __restric
 
 }  // namespace
 
-cudaError_t launch_router_simt(const float* x, const float* wr, int64_t T, int N, int d, float* out, cudaStream_t s) {
+cudaError_t launch_router_simt(const void* x, const void* wr, int dtype, int64_t T, int N, int d, float* out,
+                               cudaStream_t s) {
     const int64_t warps = T * N;
     if (warps == 0) return cudaSuccess;
-    router_simt_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, s>>>(x, wr, T, N, d, out);
+    const unsigned grid = (unsigned)((warps + 7) / 8);
+    if (dtype == EXFOLD_BF16)
+        router_simt_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(x),
+                                                reinterpret_cast<const __nv_bfloat16*>(wr), T, N, d, out);
+    else
+        router_simt_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const float*>(x), reinterpret_cast<const float*>(wr), T,
+                                                N, d, out);
     count_launch();
     return cudaGetLastError();
 }

@@ -357,11 +357,12 @@ def test_host_buffer_entry_points():
 
 
 # ------------------------------------------------------------------ router scores (input of Eq. 2)
-@pytest.mark.parametrize("dtype,N,T", [("bf16", 16, 300), ("bf16", 8, 129), ("bf16", 200, 1000), ("bf16", 6, 77),
-                                       ("f32", 8, 64)])
+@pytest.mark.parametrize("dtype,N,T", [("bf16", 16, 300), ("bf16", 8, 129), ("bf16", 200, 1000), ("bf16", 6, 277),
+                                       ("bf16", 6, 77), ("bf16", 128, 64), ("f32", 8, 64)])
 def test_router_logits_match_oracle(dtype, N, T):
     """logits = x W_r^T on the tensor cores (bf16) / fp32 dot products: within 1e-4 of the largest score.
-    N = 8 and 6 end inside the first 32-column chunk (6: rows not 16-byte aligned), N = 200 spans seven."""
+    N = 8 and 6 end inside the first 32-column chunk (6: rows not 16-byte aligned), N = 200 spans seven; batches of
+    at most 128 tokens take the dot-product kernel also for bf16."""
     cfg = small_bf16(n_experts=N, top_k=2, dtype=dtype, prefill_tokens=T, hidden=256 if dtype == "bf16" else 128)
     ex = Case(cfg).ex
     dev = torch.device("cuda:0")
