@@ -444,6 +444,61 @@ def run_ours(args, rank, world):
         dist.destroy_process_group()
 
 
+def run_decode_sweep(args):
+    """Decode batch x pool sweep on one workload's layer (default: the Qwen3-shaped one): us/layer, effective pool,
+    GB/s on the pool's weight bytes, speed-up over the unfolded layer (M = N). One GPU, one JSON line."""
+    import torch
+    from paper_2608_24938_b200 import binding as ex
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    cfg = si.CONFIGS[args.workload]
+    peaks, peak_src = load_peaks()
+    K, N, d, I = cfg.top_k, cfg.n_experts, cfg.hidden, cfg.inter
+    batches = [b for b in (1, 8, 32, 128, 256) if b * K <= 4096]
+    pools = sorted({m for m in (8, 16, 32, 64, 128) if m < N} | {N})
+    inp = build_inputs(cfg, 8, max(batches))
+    g = lambda t: t.to(dev)
+    wg, wu, wd = g(inp["wg"]), g(inp["wu"]), g(inp["wd"])
+    tables = ex.make_tables(*[g(t) for t in inp["tables"]])
+    layer = ex.make_layer(N, cfg.n_shared, d, I, K, cfg.dtype)
+    ws = ex.alloc_workspace(layer, max(batches), K)
+    flush_buf = torch.zeros(128 << 20, dtype=torch.int32, device=dev)
+    el = 2 if cfg.dtype == "bf16" else 4
+    table = []
+    for B in batches:
+        xd, lgd = g(inp["xd"][:B].contiguous()), g(inp["lgd"][:B].contiguous())
+        yd = torch.empty((B, d), dtype=wg.dtype, device=dev)
+        meta = dict(pool_size=torch.zeros(1, dtype=torch.int32, device=dev))
+        row = {}
+        for M in pools:
+            ts = []
+            for it in range(args.steps + max(args.warmup, 3)):
+                torch.sum(flush_buf)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                ex.exfold_moe_decode(layer, xd, lgd, wg, wu, wd, tables, M, yd, ws, meta=meta)
+                e1.record()
+                torch.cuda.synchronize()
+                if it >= max(args.warmup, 3):
+                    ts.append(e0.elapsed_time(e1))
+            assert ex.exfold_device_status(ws) == 0
+            us = float(np.mean(ts)) * 1e3
+            pool = int(meta["pool_size"].item())
+            byts = (pool + cfg.n_shared) * 3.0 * d * I * el
+            row[M] = {"us": us, "pool": pool, "gbs": byts / (us * 1e-6) / 1e9}
+        for M in pools:
+            r = row[M]
+            table.append({"B": B, "M": M, "effective_pool": r["pool"], "us_per_layer": round(r["us"], 2),
+                          "gbs_on_pool_bytes": round(r["gbs"], 1),
+                          "frac_of_measured_hbm": round(r["gbs"] / peaks["hbm_gbs"], 3),
+                          "speedup_vs_unfolded": round(row[N]["us"] / r["us"], 3)})
+    print(json.dumps({"metric": "decode sweep: us/layer and GB/s on pool weight bytes", "workload": cfg.name,
+                      "unit": "us/layer", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+                      "dtype": cfg.dtype, "data": "synthetic", "peaks": {"source": peak_src, **peaks},
+                      "l2": "512 MiB buffer read between calls", "table": table}), flush=True)
+
+
 def run_reference(args, rank, world):
     """The reference arm of this benchmark is the CPU oracle (the paper ships no code to install)."""
     if rank != 0:
@@ -495,13 +550,18 @@ def main():
     ap.add_argument("--layers", type=int, default=0,
                     help="also time a stack of this many decode layers (router scores + folded decode layer each), "
                          "launched on the stream and replayed as one CUDA graph")
+    ap.add_argument("--decode-sweep", action="store_true",
+                    help="instead of the benchmark line: decode batch x pool sweep on --workload (one GPU)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-flop-budget", type=float, default=3e11,
                     help="flop of oracle work in the cpu-baseline sample (about 10-30 s of CPU time)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
-    if args.impl == "reference":
+    if args.decode_sweep:
+        if rank == 0:
+            run_decode_sweep(args)
+    elif args.impl == "reference":
         run_reference(args, rank, world)
     else:
         run_ours(args, rank, world)
