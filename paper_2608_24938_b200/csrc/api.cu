@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cmath>
 #include <cstring>
 
@@ -156,19 +157,29 @@ EncodeTiledFn encode_fn() {
 
 constexpr int kMaxHostChunks = 4;  // host-buffer prefill: chunks of >= 2048 tokens in flight
 
-// bf16 matrix [rows][cols] row-major; box = box_rows x 64 columns (128 bytes), 128-byte swizzle
+// bf16 matrix [rows][cols] row-major; box = box_rows x kGemmBK columns, swizzle as wide as a box row
 bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t box[2] = {(cuuint32_t)kGemmBK, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, kGemmBK == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
+
+// EXFOLD_PAIR_GEMM=0 keeps prefill on the one-CTA kernel; =2 takes the CTA-pair kernel whenever a pair can exist
+// (the parity tests run both kernels on small inputs this way); unset or 1: the choice below. Read at every call.
+int pair_gemm_mode() {
+    const char* e = getenv("EXFOLD_PAIR_GEMM");
+    const int mode = e ? atoi(e) : 1;
+    return mode < 0 || mode > 2 ? 1 : mode;
+}
+bool force_single_cta() { return pair_gemm_mode() == 0; }
 
 int sm_count() {
     static int n = 0;
@@ -307,13 +318,25 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     const bool bf16 = l.dtype == EXFOLD_BF16;
     const bool direct = bf16 && Kp == 1 && l.n_shared == 0;  // every token is written exactly once
 
-    CUtensorMap tm_xs, tm_x, tm_wg, tm_wu, tm_h, tm_wd;
+    CUtensorMap tm_xs, tm_x, tm_wg, tm_wu, tm_h, tm_wd, tm_wd_half;
+    // A GEMM with enough work runs every group's row tiles two at a time on CTA pairs (gemm_pair.cu: a third less
+    // operand traffic per SM, a deeper ring) and leaves only a group's odd last tile to the one-CTA kernel. The pair
+    // pass pays when (a) few tiles are odd ones (about one per two groups) and (b) the pair items fill the 74 CTA
+    // pairs for several rounds; otherwise the one-CTA kernel alone is faster (measured: Mixtral shape, 4096 tokens,
+    // GEMM-2 3.5 rounds +13 %; Qwen3 shape, one tile in five odd, +4 to +8 %).
+    const int64_t tiles_est = Rtot / kTileM + G / 2;
+    const int64_t pair_est = std::max<int64_t>(0, (tiles_est - G / 2) / 2);
+    const bool pairs_ok = bf16 && kGemmBK == 64 && !force_single_cta() && (int64_t)(G / 2) * 8 <= tiles_est;
+    const int n_pairs_hw = std::max(1, sm_count() / 2);
+    const bool pairs_all = bf16 && kGemmBK == 64 && pair_gemm_mode() == 2 && Rtot >= 2 * kTileM;
+    const bool pairs1 = pairs_all || (pairs_ok && pair_est * ((I + 127) / 128) >= 8 * (int64_t)n_pairs_hw);
+    const bool pairs2 = pairs_all || (pairs_ok && pair_est * ((d + 255) / 256) >= 8 * (int64_t)n_pairs_hw);
     if (bf16) {
         const uint64_t E = (uint64_t)G;
         bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)R, d, 128) && make_tmap(&tm_x, x, (uint64_t)T, d, 128) &&
                   make_tmap(&tm_wg, w_gate, E * I, d, 128) && make_tmap(&tm_wu, w_up, E * I, d, 128) &&
                   make_tmap(&tm_h, at<char>(ws, pl.H), (uint64_t)Rtot, I, 128) &&
-                  make_tmap(&tm_wd, w_down, E * d, I, 256);
+                  make_tmap(&tm_wd, w_down, E * d, I, 256) && make_tmap(&tm_wd_half, w_down, E * d, I, 128);
         if (!ok) return EXFOLD_ERR_CUDA;
     }
 
@@ -353,15 +376,33 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
         g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
         const int64_t max_tiles = Rtot / kTileM + G;
         int grid1 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
-        { ProfScope ps(3, s); EXFOLD_CUDA(launch_grouped_gemm1(g, grid1, s)); }
-        g.tm_a = tm_h; g.tm_b0 = tm_wd; g.n_ntiles = (d + 255) / 256;
+        {
+            ProfScope ps(3, s);
+            if (pairs1) {
+                EXFOLD_CUDA(launch_grouped_gemm1_pair(g, grid1, s));
+                g.odd_only = 1;
+                grid1 = (int)std::min<int64_t>(sm_count(), (int64_t)G * g.n_ntiles);
+            }
+            EXFOLD_CUDA(launch_grouped_gemm1(g, grid1, s));
+            g.odd_only = 0;
+        }
+        g.tm_a = tm_h; g.tm_b0 = tm_wd; g.tm_b1 = tm_wd_half; g.n_ntiles = (d + 255) / 256;
         // K' = 1 without a shared expert: every token is written once, straight into y. Otherwise each
         // route's weighted output goes to O (bf16, sorted rows) and the combine kernel sums per token.
         g.y32 = nullptr;
         g.y = direct ? reinterpret_cast<__nv_bfloat16*>(y) : at<__nv_bfloat16>(ws, pl.obuf);
         g.store_rows = direct ? 0 : 1;
         int grid2 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
-        { ProfScope ps(4, s); EXFOLD_CUDA(launch_grouped_gemm2(g, grid2, s)); }
+        {
+            ProfScope ps(4, s);
+            if (pairs2) {
+                EXFOLD_CUDA(launch_grouped_gemm2_pair(g, grid2, s));
+                g.odd_only = 1;
+                grid2 = (int)std::min<int64_t>(sm_count(), (int64_t)G * g.n_ntiles);
+            }
+            EXFOLD_CUDA(launch_grouped_gemm2(g, grid2, s));
+            g.odd_only = 0;
+        }
         if (!direct) {
             ProfScope ps(5, s);
             EXFOLD_CUDA(launch_combine_rows(at<__nv_bfloat16>(ws, pl.obuf), cp.inv_pos, T, Kp, d, l.n_shared,

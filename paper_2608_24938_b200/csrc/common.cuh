@@ -22,6 +22,12 @@ constexpr int kMaxExperts = 256;  // routed experts
 constexpr int kMaxTopK = 32;
 constexpr int kMaxGroups = kMaxExperts + 1;  // + shared expert
 constexpr int kTileM = 128;                  // token rows per prefill GEMM tile
+#ifndef EXFOLD_BK
+#define EXFOLD_BK 64
+#endif
+// K elements per pipeline stage of the tensor-core GEMMs: 64 (128-byte rows, 128-byte swizzle) or 32 (64-byte rows,
+// 64-byte swizzle: half the bytes per stage, so twice as many stages fit in shared memory)
+constexpr int kGemmBK = EXFOLD_BK;
 constexpr int kMaxDecodeBatch = 256;
 constexpr int kMaxCtas = 160;                // persistent grids never exceed this (148 SMs on B200)
 
@@ -245,7 +251,7 @@ struct GroupedGemmParams {
     CUtensorMap tm_a;    // GEMM-1: gathered rows Xs [R][d]; GEMM-2: H [Rtot][I]
     CUtensorMap tm_a2;   // GEMM-1: x [T][d] for the shared expert's rows
     CUtensorMap tm_b0;   // GEMM-1: W_gate as [(E*I)][d]; GEMM-2: W_down as [(E*d)][I]
-    CUtensorMap tm_b1;   // GEMM-1: W_up
+    CUtensorMap tm_b1;   // GEMM-1: W_up; GEMM-2 on CTA pairs: W_down with 128-row boxes (each CTA stages half a tile)
     const int32_t* offsets;     // [G+1]
     const int32_t* work_start;  // [G+1] prefix of row tiles
     int G;                      // groups (N + n_shared)
@@ -266,9 +272,14 @@ struct GroupedGemmParams {
     int store_rows;             // 1: y is the per-route buffer O[row][d] that the combine kernel sums
     float* o32;                 // GEMM-2, calibration: unweighted fp32 outputs O32[row][d] (null: the epilogues above)
     int x_rows;                 // GEMM-1: rows of x; a group that reads x directly starts at row (row0 - R) % x_rows
+    int odd_only;               // 1: only each group's last row tile, and only if its tile count is odd (the rest ran on CTA pairs)
     DeviceStatus* status;
 };
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s);
 cudaError_t launch_grouped_gemm2(const GroupedGemmParams& p, int grid, cudaStream_t s);
+// Prefill on CTA pairs: every group's row tiles two at a time (a last odd tile is left to the kernels above with
+// odd_only = 1). GEMM-2 needs tm_b1 = W_down with 128-row boxes. No grp_expert, no K split, y32 = null.
+cudaError_t launch_grouped_gemm1_pair(const GroupedGemmParams& p, int grid, cudaStream_t s);
+cudaError_t launch_grouped_gemm2_pair(const GroupedGemmParams& p, int grid, cudaStream_t s);
 
 }  // namespace exfold

@@ -26,14 +26,24 @@ namespace exfold {
 namespace {
 
 constexpr int kTraceKb = 1280;  // trace builds: k-blocks logged (table 3 of the trace array holds 2 x 1280 words)
-constexpr int kBK = 64;                       // K elements per stage: 128 bytes = one swizzle row
-constexpr int kStages = 4;
-constexpr int kMaxStages = 6;  // decode loads a shorter A box per stage and fits more stages
+constexpr int kBK = kGemmBK;                  // K elements per stage: one swizzle row (128 or 64 bytes)
+#ifndef EXFOLD_STAGES
+#define EXFOLD_STAGES (EXFOLD_BK == 64 ? 4 : 9)
+#endif
+constexpr int kStages = EXFOLD_STAGES;
+constexpr int kMaxStages = kBK == 64 ? 6 : 12;  // decode loads a shorter A box per stage and fits more stages
 constexpr int kATileBytes = kTileM * kBK * 2;  // 16 KB
 constexpr int kBTileBytes = 256 * kBK * 2;     // 32 KB
 constexpr int kStageBytes = kATileBytes + kBTileBytes;
 constexpr int kGemmSmem = kStages * kStageBytes + 1024;
-constexpr int kGemmThreads = 192;
+#ifndef EXFOLD_PRODUCERS
+#define EXFOLD_PRODUCERS (EXFOLD_BK == 64 ? 2 : 3)
+#endif
+// One thread's loop {wait for the stage, expect_tx, 2-3 TMA issues} takes ~600-700 cycles: longer than the 512
+// cycles the tensor pipe needs for a k-block. The k-blocks are therefore dealt round-robin over kProducers
+// one-thread producers in warps of their own (warp 0 and the warps after the epilogue warps).
+constexpr int kProducers = EXFOLD_PRODUCERS;
+constexpr int kGemmThreads = 192 + 32 * (kProducers - 1);
 constexpr int kTmemCols = 512;
 
 struct WorkItem {
@@ -42,7 +52,8 @@ struct WorkItem {
 
 // Work index -> (group, row tile, column tile, K part). Order: group, column tile, row tile, K part
 // (fastest), so CTAs running together share weight tiles through L2.
-__device__ __forceinline__ WorkItem decode_work(int w_all, int G, int nt, int ks, const int* s_off, const int* s_ws) {
+__device__ __forceinline__ WorkItem decode_work(int w_all, int G, int nt, int ks, const int* s_off, const int* s_ws,
+                                                int odd_only = 0) {
     const int w = ks == 1 ? w_all : w_all / ks;
     int lo = 0, hi = G;  // find g with s_ws[g]*nt <= w < s_ws[g+1]*nt
     while (hi - lo > 1) {
@@ -60,7 +71,9 @@ __device__ __forceinline__ WorkItem decode_work(int w_all, int G, int nt, int ks
     const int m_idx = local % tiles;
     it.m_idx = m_idx;
     it.n_idx = local / tiles;
-    it.row0 = s_off[lo] + m_idx * kTileM;
+    // odd_only: the group's one item is its LAST row tile (the tiles before it ran two at a time on CTA pairs)
+    const int first = odd_only ? (s_off[lo + 1] - s_off[lo] - 1) / kTileM : 0;
+    it.row0 = s_off[lo] + (first + m_idx) * kTileM;
     const int left = s_off[lo + 1] - it.row0;
     it.rows = left < kTileM ? left : kTileM;
     return it;
@@ -133,6 +146,27 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (!DEC && p.odd_only) {
+        // work table of the odd-tile pass: one row tile for every group whose tile count is odd
+        if (warp == 0) {
+            int carry = 0;
+            for (int g0 = 0; g0 < G; g0 += 32) {
+                const int g = g0 + lane;
+                int odd = 0;
+                if (g < G) odd = ((s_off[g + 1] - s_off[g] + kTileM - 1) / kTileM) & 1;
+                int incl = odd;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += v;
+                }
+                if (g < G) s_ws[g] = carry + incl - odd;
+                carry += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (lane == 0) s_ws[G] = carry;
+        }
+        __syncthreads();
+    }
     ptx::tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
     const int nt = p.n_ntiles;
@@ -150,19 +184,20 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     // Stage geometry. Prefill: 16 KB A + 32 KB B, 4 stages (compile-time). Decode: the A box has only
     // a_rows rows (the rest of the 128-row MMA operand is whatever follows in shared memory: those
     // accumulator rows are masked), so a stage is smaller and more stages of weights are in flight.
-    const int a_bytes = DEC ? p.a_rows * 128 : kATileBytes;
+    const int a_bytes = DEC ? p.a_rows * kBK * 2 : kATileBytes;
     const int stage_bytes = DEC ? a_bytes + kBTileBytes : kStageBytes;
     const int stages = DEC ? min(kMaxStages, (kStages * kStageBytes - (kATileBytes - a_bytes)) / stage_bytes) : kStages;
     volatile int* abort_flag = &abort_s;
     if (threadIdx.x == 0) EXFOLD_TRACE_SET(kTr, 1, ptx::globaltimer_ns());
 
-    if (warp == 0) {
-        // ------------------------------------------------ TMA producer
+    if (warp == 0 || warp >= 6) {
+        // ------------------------------------------------ TMA producers (k-block c belongs to producer c % kProducers)
         if (lane == 0) {
-            int stage = 0, phase = 0;
+            const int me = warp == 0 ? 0 : warp - 5;
+            int stage = 0, phase = 0, turn = 0;
             bool ok = true;
             for (int w = w_begin; w < total && ok; w += w_stride) {
-                const WorkItem it = decode_work(w, G, nt, ks, s_off, s_ws);
+                const WorkItem it = decode_work(w, G, nt, ks, s_off, s_ws, DEC ? 0 : p.odd_only);
                 const int kb0 = it.kpart * kb_per, kb1 = min(nkb, kb0 + kb_per);
                 // per-tile constants stay in registers: the k-loop below is the latency-critical path
                 const int expert = DEC ? s_exp[it.g] : it.g;
@@ -171,26 +206,32 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                 const int arow = from_x ? (it.row0 - p.R) % p.x_rows : it.row0;
                 const int brow = MODE == 0 ? expert * p.I + it.n_idx * 128 : expert * p.d + it.n_idx * 256;
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    bool got;
-                    EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, p.status, 1));
-                    if (!got) {
-                        ok = false;
-                        break;
+                    if (turn == me) {
+                        bool got;
+                        EXFOLD_TRACE_ADD(tr_wait,
+                                         got = ptx::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, p.status, 1));
+                        if (!got) {
+                            ok = false;
+                            break;
+                        }
+                        unsigned char* a_dst = tiles + stage * stage_bytes;
+                        unsigned char* b_dst = a_dst + a_bytes;
+                        ptx::mbar_expect_tx(&full_bar[stage], stage_bytes);
+                        ptx::tma_load_2d(a_dst, tma_a, &full_bar[stage], kb * kBK, arow);
+                        ptx::tma_load_2d(b_dst, &p.tm_b0, &full_bar[stage], kb * kBK, brow);
+                        if (MODE == 0) ptx::tma_load_2d(b_dst + 128 * kBK * 2, &p.tm_b1, &full_bar[stage], kb * kBK, brow);
                     }
-                    unsigned char* a_dst = tiles + stage * stage_bytes;
-                    unsigned char* b_dst = a_dst + a_bytes;
-                    ptx::mbar_expect_tx(&full_bar[stage], stage_bytes);
-                    ptx::tma_load_2d(a_dst, tma_a, &full_bar[stage], kb * kBK, arow);
-                    ptx::tma_load_2d(b_dst, &p.tm_b0, &full_bar[stage], kb * kBK, brow);
-                    if (MODE == 0) ptx::tma_load_2d(b_dst + 128 * 128, &p.tm_b1, &full_bar[stage], kb * kBK, brow);
+                    if (++turn == kProducers) turn = 0;
                     if (++stage == stages) {
                         stage = 0;
                         phase ^= 1;
                     }
                 }
             }
-            EXFOLD_TRACE_SET(kTr, 3, tr_wait);
-            EXFOLD_TRACE_SET(kTr, 4, ptx::globaltimer_ns());
+            if (me == 0) {
+                EXFOLD_TRACE_SET(kTr, 3, tr_wait);
+                EXFOLD_TRACE_SET(kTr, 4, ptx::globaltimer_ns());
+            }
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -201,7 +242,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
 #ifdef EXFOLD_TRACE
             int kbt = 0;
 #endif
+            // This one thread's instruction stream paces the tensor pipe (a k-block is 4 MMAs = 512 pipe cycles),
+            // so the loop carries as little as possible: the descriptors' low words advance by a constant per stage
+            // (the high word never changes), and the readiness of the NEXT stage is polled before this stage's MMAs
+            // are issued, so that the poll's round trip overlaps them.
+            const uint32_t lo0 = (ptx::smem_u32(tiles) & 0x3FFFFu) >> 4;
+            const uint32_t lo_step = (uint32_t)stage_bytes >> 4, lo_b = (uint32_t)a_bytes >> 4;
+            const uint32_t desc_hi32 = (uint32_t)(ptx::make_kmajor_sw128_desc(0) >> 32);
+            uint32_t a_lo = lo0;
             bool ok = true;
+            bool ready = false;
             for (int w = w_begin; w < total && ok; w += w_stride, ++iter) {
                 const int as = iter & 1, aphase = (iter >> 1) & 1;
                 bool got;
@@ -212,33 +262,37 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                 const int kpart = ks == 1 ? 0 : w % ks;
                 const int kb0 = kpart * kb_per, kb1 = min(nkb, kb0 + kb_per);
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3));
-                    if (iter == 0 && kb == kb0) EXFOLD_TRACE_SET(kTr, 9, ptx::globaltimer_ns());
-                    if (!got) {
-                        ok = false;
-                        break;
+                    if (!ready) {
+                        EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3));
+                        if (!got) {
+                            ok = false;
+                            break;
+                        }
                     }
-                    ptx::tc_fence_after();
+                    if (iter == 0 && kb == kb0) EXFOLD_TRACE_SET(kTr, 9, ptx::globaltimer_ns());
 #ifdef EXFOLD_TRACE
-                    // one CTA of the chosen prefill GEMM logs when each k-block's operands were ready (cycles, ns)
+                    // one CTA of the chosen prefill GEMM logs when each k-block's operands were ready (cycles; the
+                    // ns timer once per 16 k-blocks, for the clock rate)
+#ifdef EXFOLD_TRACE_PAIR
+                    if (false) {
+#elif defined(EXFOLD_TRACE_TILE)
+                    if (MODE == EXFOLD_TRACE_KB_MODE && !DEC && blockIdx.x == 5 && kbt < kTraceKb && kb == kb0) {
+#else
                     if (MODE == EXFOLD_TRACE_KB_MODE && !DEC && blockIdx.x == 5 && kbt < kTraceKb) {
+#endif
                         unsigned long long* flat = &g_trace[3][0][0];
                         flat[kbt] = (unsigned long long)clock64();
-                        flat[kTraceKb + kbt] = ptx::globaltimer_ns();
+                        if ((kbt & 15) == 0) flat[kTraceKb + kbt] = ptx::globaltimer_ns();
                         ++kbt;
                     }
 #endif
-                    const uint32_t a_addr = ptx::smem_u32(tiles + stage * stage_bytes);
-                    const uint64_t adesc = ptx::make_kmajor_sw128_desc(a_addr);
-                    const uint64_t bdesc = ptx::make_kmajor_sw128_desc(a_addr + a_bytes);
-#pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k)
-                        ptx::umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-                    ptx::umma_commit(&empty_bar[stage]);
-                    if (++stage == stages) {
-                        stage = 0;
-                        phase ^= 1;
-                    }
+                    const int ns = stage + 1 == stages ? 0 : stage + 1;
+                    const int nphase = ns == 0 ? phase ^ 1 : phase;
+                    ready = ptx::umma_kblock_bf16(d_tmem, a_lo, a_lo + lo_b, desc_hi32, idesc, kb > kb0 ? 1u : 0u,
+                                                  &empty_bar[stage], &full_bar[ns], nphase);
+                    a_lo = ns == 0 ? lo0 : a_lo + lo_step;
+                    stage = ns;
+                    phase = nphase;
                 }
                 if (ok) ptx::umma_commit(&tfull_bar[as]);
             }
@@ -254,7 +308,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         int iter = 0;
         for (int w = w_begin; w < total; w += w_stride, ++iter) {
             const int as = iter & 1, aphase = (iter >> 1) & 1;
-            const WorkItem it = decode_work(w, G, nt, ks, s_off, s_ws);
+            const WorkItem it = decode_work(w, G, nt, ks, s_off, s_ws, DEC ? 0 : p.odd_only);
             // lane 0 waits; the warp takes one decision, so the warp-wide TMEM loads below stay convergent
             int ok = 1;
             if (lane == 0) {

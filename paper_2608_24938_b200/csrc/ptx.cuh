@@ -132,6 +132,133 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
         "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// One k-block of the main loop in a single instruction sequence: poll `next_full` (the NEXT stage's operands), issue
+// kGemmBK/16 K=16 MMAs on this stage's operands (descriptor low words advance by 32 bytes = 2 per MMA;
+// `desc_hi` is the shared high word), commit to `empty`, and only then read the poll's predicate, so that the
+// poll's round trip overlaps the MMA issue. Returns whether the next stage was already complete.
+__device__ __forceinline__ bool umma_kblock_bf16(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                                 uint32_t idesc, uint32_t acc_first, uint64_t* empty,
+                                                 uint64_t* next_full, uint32_t next_parity) {
+    uint32_t ready;
+    asm volatile(
+        "{\n"
+        ".reg .pred pr, pa;\n"
+        ".reg .b64 da, db;\n"
+        ".reg .b32 la, lb;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 pr, [%8], %9;\n"
+        "setp.ne.b32 pa, %6, 0;\n"
+        "mov.b64 da, {%2, %4};\n"
+        "mov.b64 db, {%3, %4};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, pa;\n"
+        "add.u32 la, %2, 2;\n"
+        "add.u32 lb, %3, 2;\n"
+        "mov.b64 da, {la, %4};\n"
+        "mov.b64 db, {lb, %4};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, 1;\n"
+#if EXFOLD_BK == 64
+        "add.u32 la, %2, 4;\n"
+        "add.u32 lb, %3, 4;\n"
+        "mov.b64 da, {la, %4};\n"
+        "mov.b64 db, {lb, %4};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, 1;\n"
+        "add.u32 la, %2, 6;\n"
+        "add.u32 lb, %3, 6;\n"
+        "mov.b64 da, {la, %4};\n"
+        "mov.b64 db, {lb, %4};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, 1;\n"
+#endif
+        "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%7];\n"
+        "selp.b32 %0, 1, 0, pr;\n"
+        "}\n"
+        : "=r"(ready)
+        : "r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc_first), "r"(smem_u32(empty)),
+          "r"(smem_u32(next_full)), "r"(next_parity)
+        : "memory");
+    return ready != 0;
+}
+// ------------------------------------------------------------------ CTA pairs (cta_group::2)
+// A cluster of two CTAs issues MMAs that span both CTAs' tensor cores and tensor memory: each CTA stages its own
+// 128 A rows and its half of B at the same shared-memory offsets, the leader (cluster rank 0) issues.
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;  // clears the CTA-rank bit of a shared::cluster address: CTA 0's copy
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {  // same warp in both CTAs
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {  // same warp in both CTAs
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// 2-D tiled load into this CTA's shared memory; the bytes are counted on the LEADER CTA's barrier at `bar`'s offset
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* m, uint64_t* bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(m), "r"(smem_u32(bar) & kPeerBitMask), "r"(c0), "r"(c1)
+        : "memory");
+}
+// Arrive on the barrier at `bar`'s offset in every CTA of `cta_mask` once the MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mask) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(smem_u32(bar)), "h"(cta_mask)
+        : "memory");
+}
+// Arrive on the leader CTA's barrier at `bar`'s offset (from either CTA of the pair)
+__device__ __forceinline__ void mbar_arrive_leader(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(smem_u32(bar) & kPeerBitMask) : "memory");
+}
+// The pair form of umma_kblock_bf16 (K = 64 per stage): four M256 MMAs over both CTAs, the commit frees the stage in
+// both CTAs (`empty` at the same offset in each).
+__device__ __forceinline__ bool umma_kblock_bf16_pair(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                                      uint32_t idesc, uint32_t acc_first, uint64_t* empty,
+                                                      uint64_t* next_full, uint32_t next_parity) {
+    uint32_t ready;
+    const uint16_t both = 3;
+    asm volatile(
+        "{\n"
+        ".reg .pred pr, pa;\n"
+        ".reg .b64 da, db;\n"
+        ".reg .b32 la, lb;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 pr, [%8], %9;\n"
+        "setp.ne.b32 pa, %6, 0;\n"
+        "mov.b64 da, {%2, %4};\n"
+        "mov.b64 db, {%3, %4};\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], da, db, %5, pa;\n"
+        "add.u32 la, %2, 2;\n"
+        "add.u32 lb, %3, 2;\n"
+        "mov.b64 da, {la, %4};\n"
+        "mov.b64 db, {lb, %4};\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], da, db, %5, 1;\n"
+        "add.u32 la, %2, 4;\n"
+        "add.u32 lb, %3, 4;\n"
+        "mov.b64 da, {la, %4};\n"
+        "mov.b64 db, {lb, %4};\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], da, db, %5, 1;\n"
+        "add.u32 la, %2, 6;\n"
+        "add.u32 lb, %3, 6;\n"
+        "mov.b64 da, {la, %4};\n"
+        "mov.b64 db, {lb, %4};\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], da, db, %5, 1;\n"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%7], %10;\n"
+        "selp.b32 %0, 1, 0, pr;\n"
+        "}\n"
+        : "=r"(ready)
+        : "r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc_first), "r"(smem_u32(empty)),
+          "r"(smem_u32(next_full)), "r"(next_parity), "h"(both)
+        : "memory");
+    return ready != 0;
+}
 // Arrive on `bar` once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -163,17 +290,18 @@ __device__ __forceinline__ void tmem_ld_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// Shared-memory matrix descriptor for a K-major bf16 tile stored as rows of 64 elements (128 bytes)
-// with the 128-byte swizzle TMA applies (SWIZZLE_128B): 8-row groups are 1024 bytes apart. The
-// tile base must be 1024-byte aligned. Advancing by 16 elements along K adds 32 bytes (>>4 = 2)
+// Shared-memory matrix descriptor for a K-major bf16 tile stored as rows of kGemmBK elements (128 or 64 bytes)
+// with the swizzle TMA applies (SWIZZLE_128B / SWIZZLE_64B): 8-row groups are 8 rows apart (1024 / 512 bytes).
+// The tile base must be aligned to that group size. Advancing by 16 elements along K adds 32 bytes (>>4 = 2)
 // to the start-address field.
 __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
+    constexpr uint32_t group_bytes = 8u * kGemmBK * 2u;
     uint64_t desc = 0;
     desc |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);   // start address, bits [0,14)
     desc |= (uint64_t)0 << 16;                         // leading byte offset: unused for swizzled K-major
-    desc |= (uint64_t)(1024u >> 4) << 32;              // stride byte offset between 8-row groups
+    desc |= (uint64_t)(group_bytes >> 4) << 32;        // stride byte offset between 8-row groups
     desc |= (uint64_t)1 << 46;                         // descriptor version for sm_100
-    desc |= (uint64_t)2 << 61;                         // layout type: SWIZZLE_128B
+    desc |= (uint64_t)(kGemmBK == 64 ? 2 : 4) << 61;   // layout type: SWIZZLE_128B = 2, SWIZZLE_64B = 4
     return desc;
 }
 

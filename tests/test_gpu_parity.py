@@ -182,6 +182,36 @@ def test_bf16_several_tiles_and_ragged_tail():
     check_output(got["y"], ref["y"], "bf16")
 
 
+@pytest.mark.parametrize("shape", ["skewed", "shared", "top1"])
+def test_prefill_on_cta_pairs_matches_oracle_and_the_one_cta_kernel(shape, monkeypatch):
+    """EXFOLD_PAIR_GEMM=2 runs every pair of row tiles of a group on the CTA-pair kernel and the odd last tiles on the
+    one-CTA kernel, whatever the size; =0 keeps everything on the one-CTA kernel. Both must match the oracle, and
+    each other to the last bit (the same products are accumulated in the same order)."""
+    if shape == "skewed":    # groups of 0, 1, 2, 3, ... row tiles, ragged last tiles, K and N tails
+        cfg = small_bf16(n_experts=8, hidden=512, inter=832, top_k=2, prefill_tokens=1500, logits="zipf", zipf_s=1.5)
+        Kps = (1, 2)
+    elif shape == "shared":  # the shared expert's group reads x in place: 7 tiles = 3 pairs + an odd tile
+        cfg = small_bf16(n_experts=6, n_shared=1, hidden=320, inter=448, top_k=3, prefill_tokens=777, logits="normal")
+        Kps = (2,)
+    else:                    # K' = 1 without a shared expert: GEMM-2 writes y directly
+        cfg = small_bf16(n_experts=4, hidden=256, inter=256, top_k=2, prefill_tokens=1024, logits="normal")
+        Kps = (1,)
+    case = Case(cfg)
+    for Kp in Kps:
+        ref = case.oracle_prefill(Kp)
+        monkeypatch.setenv("EXFOLD_PAIR_GEMM", "2")
+        got_pair = case.run_prefill(Kp)
+        monkeypatch.setenv("EXFOLD_PAIR_GEMM", "0")
+        got_one = case.run_prefill(Kp)
+        monkeypatch.delenv("EXFOLD_PAIR_GEMM")
+        counts = np.diff(ref["offsets"])
+        assert counts.max() >= 256          # at least one whole pair of row tiles
+        check_prefill_meta(got_pair, ref)
+        check_output(got_pair["y"], ref["y"], "bf16")
+        check_output(got_one["y"], ref["y"], "bf16")
+        assert np.array_equal(got_pair["y"], got_one["y"])   # bf16 values widened to float32: exact comparison
+
+
 @pytest.mark.parametrize("T", [1, 63, 129])
 def test_bf16_odd_token_counts(T):
     cfg = small_bf16(prefill_tokens=T, decode_batch=min(T, 256))
