@@ -33,7 +33,7 @@ EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibr
            "exfold_moe_prefill_ex", "exfold_router_logits"]
 PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
                  "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
-                 "simt_combine"]
+                 "simt_combine", "gemm1_pair_pass", "gemm2_pair_pass"]
 
 
 class exfold_layer(C.Structure):

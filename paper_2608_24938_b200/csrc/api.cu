@@ -60,7 +60,7 @@ void prof_reset() {
 struct Plan {
     size_t status, ids, w, omit_src, omit_tgt, block_hist, offsets, work_start, totals, perm, row_tok, row_w,
         row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
-        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, total;
+        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, work_ctr, total;
 };
 
 bool valid_layer(const exfold_layer* l) {
@@ -95,6 +95,7 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
     p.offsets = take((G + 2) * 4);
     p.work_start = take((G + 2) * 4);
     p.totals = take(16);
+    p.work_ctr = take(16);
     p.perm = take(Rm * 4);
     p.inv_pos = take(Rm * 4);
     p.row_tok = take(Rtot * 4);
@@ -179,7 +180,6 @@ int pair_gemm_mode() {
     const int mode = e ? atoi(e) : 1;
     return mode < 0 || mode > 2 ? 1 : mode;
 }
-bool force_single_cta() { return pair_gemm_mode() == 0; }
 
 int sm_count() {
     static int n = 0;
@@ -321,16 +321,19 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     CUtensorMap tm_xs, tm_x, tm_wg, tm_wu, tm_h, tm_wd, tm_wd_half;
     // A GEMM with enough work runs every group's row tiles two at a time on CTA pairs (gemm_pair.cu: a third less
     // operand traffic per SM, a deeper ring) and leaves only a group's odd last tile to the one-CTA kernel. The pair
-    // pass pays when (a) few tiles are odd ones (about one per two groups) and (b) the pair items fill the 74 CTA
-    // pairs for several rounds; otherwise the one-CTA kernel alone is faster (measured: Mixtral shape, 4096 tokens,
-    // GEMM-2 3.5 rounds +13 %; Qwen3 shape, one tile in five odd, +4 to +8 %).
+    // pass pays when the call is large (>= 64 row tiles: its advantage grows with the kernels' duration), few tiles
+    // are odd ones (about one per two groups; at most one tile in eight) and the pair items fill the 74 CTA pairs
+    // for several rounds; otherwise the one-CTA kernel alone is faster (measured: Mixtral shape, 4096 tokens = 36
+    // tiles: +1.5 %; Qwen3 shape, one tile in five odd: +4 to +8 %; Mixtral shape 8192 / 16384 / 32768 tokens:
+    // -7 / -9 / -15 %; GLM shape: -6 %).
     const int64_t tiles_est = Rtot / kTileM + G / 2;
     const int64_t pair_est = std::max<int64_t>(0, (tiles_est - G / 2) / 2);
-    const bool pairs_ok = bf16 && kGemmBK == 64 && !force_single_cta() && (int64_t)(G / 2) * 8 <= tiles_est;
+    const int mode = pair_gemm_mode();
+    const bool pairs_ok = bf16 && kGemmBK == 64 && mode == 1 && tiles_est >= 64 && (int64_t)(G / 2) * 8 <= tiles_est;
+    const bool pairs_all = bf16 && kGemmBK == 64 && mode == 2 && Rtot >= 2 * kTileM;
     const int n_pairs_hw = std::max(1, sm_count() / 2);
-    const bool pairs_all = bf16 && kGemmBK == 64 && pair_gemm_mode() == 2 && Rtot >= 2 * kTileM;
-    const bool pairs1 = pairs_all || (pairs_ok && pair_est * ((I + 127) / 128) >= 8 * (int64_t)n_pairs_hw);
-    const bool pairs2 = pairs_all || (pairs_ok && pair_est * ((d + 255) / 256) >= 8 * (int64_t)n_pairs_hw);
+    const bool pairs1 = pairs_all || (pairs_ok && pair_est * ((I + 127) / 128) >= 6 * (int64_t)n_pairs_hw);
+    const bool pairs2 = pairs_all || (pairs_ok && pair_est * ((d + 255) / 256) >= 6 * (int64_t)n_pairs_hw);
     if (bf16) {
         const uint64_t E = (uint64_t)G;
         bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)R, d, 128) && make_tmap(&tm_x, x, (uint64_t)T, d, 128) &&
@@ -364,6 +367,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
     cp.row_w = at<float>(ws, pl.row_w); cp.row_exp = at<int32_t>(ws, pl.row_exp);
     cp.inv_pos = at<int32_t>(ws, pl.inv_pos);
+    cp.work_ctr = at<int32_t>(ws, pl.work_ctr);
     { ProfScope ps(2, s); EXFOLD_CUDA(launch_prefill_scatter(cp, s)); }
 
     if (bf16) {
@@ -379,12 +383,14 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
         {
             ProfScope ps(3, s);
             if (pairs1) {
-                EXFOLD_CUDA(launch_grouped_gemm1_pair(g, grid1, s));
+                { ProfScope pp(12, s); EXFOLD_CUDA(launch_grouped_gemm1_pair(g, grid1, s)); }
                 g.odd_only = 1;
+                g.work_ctr = cp.work_ctr;
                 grid1 = (int)std::min<int64_t>(sm_count(), (int64_t)G * g.n_ntiles);
             }
             EXFOLD_CUDA(launch_grouped_gemm1(g, grid1, s));
             g.odd_only = 0;
+            g.work_ctr = nullptr;
         }
         g.tm_a = tm_h; g.tm_b0 = tm_wd; g.tm_b1 = tm_wd_half; g.n_ntiles = (d + 255) / 256;
         // K' = 1 without a shared expert: every token is written once, straight into y. Otherwise each
@@ -396,12 +402,14 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
         {
             ProfScope ps(4, s);
             if (pairs2) {
-                EXFOLD_CUDA(launch_grouped_gemm2_pair(g, grid2, s));
+                { ProfScope pp(13, s); EXFOLD_CUDA(launch_grouped_gemm2_pair(g, grid2, s)); }
                 g.odd_only = 1;
+                g.work_ctr = cp.work_ctr + 1;
                 grid2 = (int)std::min<int64_t>(sm_count(), (int64_t)G * g.n_ntiles);
             }
             EXFOLD_CUDA(launch_grouped_gemm2(g, grid2, s));
             g.odd_only = 0;
+            g.work_ctr = nullptr;
         }
         if (!direct) {
             ProfScope ps(5, s);
