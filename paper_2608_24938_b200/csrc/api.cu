@@ -320,16 +320,16 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
 
     CUtensorMap tm_xs, tm_x, tm_wg, tm_wu, tm_h, tm_wd, tm_wd_half;
     // A GEMM with enough work runs every group's row tiles two at a time on CTA pairs (gemm_pair.cu: a third less
-    // operand traffic per SM, a deeper ring) and leaves only a group's odd last tile to the one-CTA kernel. The pair
-    // pass pays when the call is large (>= 64 row tiles: its advantage grows with the kernels' duration), few tiles
+    // operand traffic per SM, a deeper ring, the tensor pipe busy > 95 % of the main loop) and leaves only a group's
+    // odd last tile to the one-CTA kernel. The pair pass pays when the call is large (>= 48 row tiles), few tiles
     // are odd ones (about one per two groups; at most one tile in eight) and the pair items fill the 74 CTA pairs
-    // for several rounds; otherwise the one-CTA kernel alone is faster (measured: Mixtral shape, 4096 tokens = 36
-    // tiles: +1.5 %; Qwen3 shape, one tile in five odd: +4 to +8 %; Mixtral shape 8192 / 16384 / 32768 tokens:
-    // -7 / -9 / -15 %; GLM shape: -6 %).
+    // for several rounds; otherwise the one-CTA kernel alone is as fast or faster (measured against it: Mixtral shape,
+    // 4096 tokens = 36 tiles: +0.4 %; Qwen3 shape, one tile in five odd: +4 to +8 %; Mixtral shape 6144 / 8192 /
+    // 16384 / 32768 tokens: -2 / -8 / -13 / -16 %; GLM shape: -6 %).
     const int64_t tiles_est = Rtot / kTileM + G / 2;
     const int64_t pair_est = std::max<int64_t>(0, (tiles_est - G / 2) / 2);
     const int mode = pair_gemm_mode();
-    const bool pairs_ok = bf16 && kGemmBK == 64 && mode == 1 && tiles_est >= 64 && (int64_t)(G / 2) * 8 <= tiles_est;
+    const bool pairs_ok = bf16 && kGemmBK == 64 && mode == 1 && tiles_est >= 48 && (int64_t)(G / 2) * 8 <= tiles_est;
     const bool pairs_all = bf16 && kGemmBK == 64 && mode == 2 && Rtot >= 2 * kTileM;
     const int n_pairs_hw = std::max(1, sm_count() / 2);
     const bool pairs1 = pairs_all || (pairs_ok && pair_est * ((I + 127) / 128) >= 6 * (int64_t)n_pairs_hw);

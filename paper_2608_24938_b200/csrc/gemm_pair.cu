@@ -181,47 +181,77 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
             const uint32_t lo0 = (ptx::smem_u32(tiles) & 0x3FFFFu) >> 4;
             constexpr uint32_t lo_step = (uint32_t)kPStageBytes >> 4, lo_b = (uint32_t)kPATileBytes >> 4;
             const uint32_t desc_hi32 = (uint32_t)(ptx::make_kmajor_sw128_desc(0) >> 32);
-            uint32_t a_lo = lo0;
             int stage = 0, phase = 0, iter = 0;
             bool ok = true, ready = false;
+            static_assert(kPStages == 6, "the k-loop below is written out for six ring stages");
 #ifdef EXFOLD_TRACE
             int kbt = 0;
+            long long n_polls = 0, n_ready = 0;
 #endif
             for (int w = w_begin; w < total && ok; w += w_stride, ++iter) {
                 const int as = iter & 1, aphase = (iter >> 1) & 1;
                 if (!ptx::mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag, p.status, 2)) break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + as * 256;
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (!ready && !ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3)) {
-                        ok = false;
-                        break;
-                    }
+                // The k-loop is written out once per ring stage (switch into the stage the ring stands at): this
+                // thread's instruction stream paces the tensor pipe, and with the stage a compile-time constant a
+                // k-block costs it the MMA sequence, one compare and one branch.
+                int kb = 0;
+#define EXFOLD_PAIR_KBLOCK(S)                                                                                      \
+    {                                                                                                               \
+        constexpr int NS = (S) + 1 == kPStages ? 0 : (S) + 1;                                                       \
+        const uint32_t nphase = NS == 0 ? phase ^ 1 : phase;                                                        \
+        if (!ready && !ptx::mbar_wait(&full_bar[S], phase, abort_flag, p.status, 3)) {                              \
+            ok = false;                                                                                             \
+            break;                                                                                                  \
+        }                                                                                                           \
+        EXFOLD_PAIR_TRACE_KB();                                                                                     \
+        ready = ptx::umma_kblock_bf16_pair(d_tmem, lo0 + (S) * lo_step, lo0 + (S) * lo_step + lo_b, desc_hi32,    \
+                                           idesc, kb > 0 ? 1u : 0u, &empty_bar[S], &full_bar[NS], nphase);          \
+        if (NS == 0) phase ^= 1;                                                                                    \
+        if (++kb == nkb) {                                                                                          \
+            stage = NS;                                                                                             \
+            break;                                                                                                  \
+        }                                                                                                           \
+    }
 #ifdef EXFOLD_TRACE
-                    // the leader of one pair logs when each k-block's operands were ready (cycles; ns every 16th)
-                    if (MODE == EXFOLD_TRACE_KB_MODE && blockIdx.x == 10 && kbt < 1280) {
+                // the leader of one pair logs when each k-block's (with EXFOLD_TRACE_TILE: item's) operands were ready
 #ifdef EXFOLD_TRACE_TILE
-                        if (kb == 0)
+#define EXFOLD_PAIR_TRACE_COND (kb == 0)
+#else
+#define EXFOLD_PAIR_TRACE_COND true
 #endif
-                        {
-                            unsigned long long* flat = &g_trace[3][0][0];
-                            flat[kbt] = (unsigned long long)clock64();
-                            if ((kbt & 15) == 0) flat[1280 + kbt] = ptx::globaltimer_ns();
-                            ++kbt;
-                        }
+#define EXFOLD_PAIR_TRACE_KB()                                                                       \
+    do {                                                                                             \
+        n_polls += 1;                                                                                \
+        n_ready += ready ? 1 : 0;                                                                    \
+        if (MODE == EXFOLD_TRACE_KB_MODE && blockIdx.x == 10 && kbt < 1280 && EXFOLD_PAIR_TRACE_COND) { \
+            unsigned long long* flat = &g_trace[3][0][0];                                            \
+            flat[kbt] = (unsigned long long)clock64();                                               \
+            if ((kbt & 15) == 0) flat[1280 + kbt] = ptx::globaltimer_ns();                           \
+            ++kbt;                                                                                   \
+        }                                                                                            \
+    } while (0)
+#else
+#define EXFOLD_PAIR_TRACE_KB() ((void)0)
+#endif
+                while (ok && kb < nkb) {
+                    switch (stage) {
+                        case 0: EXFOLD_PAIR_KBLOCK(0)
+                        case 1: EXFOLD_PAIR_KBLOCK(1)
+                        case 2: EXFOLD_PAIR_KBLOCK(2)
+                        case 3: EXFOLD_PAIR_KBLOCK(3)
+                        case 4: EXFOLD_PAIR_KBLOCK(4)
+                        default: EXFOLD_PAIR_KBLOCK(5)
                     }
-#endif
-                    const int ns = stage + 1 == kPStages ? 0 : stage + 1;
-                    const int nphase = ns == 0 ? phase ^ 1 : phase;
-                    // polls the next stage, issues this stage's four MMAs, frees the stage in both CTAs
-                    ready = ptx::umma_kblock_bf16_pair(d_tmem, a_lo, a_lo + lo_b, desc_hi32, idesc, kb > 0 ? 1u : 0u,
-                                                       &empty_bar[stage], &full_bar[ns], nphase);
-                    a_lo = ns == 0 ? lo0 : a_lo + lo_step;
-                    stage = ns;
-                    phase = nphase;
+                    if (kb < nkb) stage = 0;  // fell through the last stage: the ring wraps
                 }
+#undef EXFOLD_PAIR_KBLOCK
+#undef EXFOLD_PAIR_TRACE_KB
                 if (ok) ptx::umma_commit_pair(&tfull_bar[as], 3);
             }
+            EXFOLD_TRACE_SET(MODE, 12, n_polls);  // k-blocks issued / of which the next stage was already complete
+            EXFOLD_TRACE_SET(MODE, 13, n_ready);
         }
         __syncwarp();
     } else {

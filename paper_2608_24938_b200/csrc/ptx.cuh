@@ -132,8 +132,8 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
         "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// One k-block of the main loop in a single instruction sequence: poll `next_full` (the NEXT stage's operands), issue
-// kGemmBK/16 K=16 MMAs on this stage's operands (descriptor low words advance by 32 bytes = 2 per MMA;
+// One k-block of the main loop in a single instruction sequence: issue kGemmBK/16 K=16 MMAs on this stage's operands,
+// with a poll of `next_full` (the NEXT stage's operands) before the last of them (descriptor low words advance by 32 bytes = 2 per MMA;
 // `desc_hi` is the shared high word), commit to `empty`, and only then read the poll's predicate, so that the
 // poll's round trip overlaps the MMA issue. Returns whether the next stage was already complete.
 __device__ __forceinline__ bool umma_kblock_bf16(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
@@ -145,7 +145,6 @@ __device__ __forceinline__ bool umma_kblock_bf16(uint32_t tmem_d, uint32_t a_lo,
         ".reg .pred pr, pa;\n"
         ".reg .b64 da, db;\n"
         ".reg .b32 la, lb;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 pr, [%8], %9;\n"
         "setp.ne.b32 pa, %6, 0;\n"
         "mov.b64 da, {%2, %4};\n"
         "mov.b64 db, {%3, %4};\n"
@@ -154,6 +153,9 @@ __device__ __forceinline__ bool umma_kblock_bf16(uint32_t tmem_d, uint32_t a_lo,
         "add.u32 lb, %3, 2;\n"
         "mov.b64 da, {la, %4};\n"
         "mov.b64 db, {lb, %4};\n"
+#if EXFOLD_BK != 64
+        "mbarrier.try_wait.parity.shared::cta.b64 pr, [%8], %9;\n"
+#endif
         "tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, 1;\n"
 #if EXFOLD_BK == 64
         "add.u32 la, %2, 4;\n"
@@ -165,6 +167,7 @@ __device__ __forceinline__ bool umma_kblock_bf16(uint32_t tmem_d, uint32_t a_lo,
         "add.u32 lb, %3, 6;\n"
         "mov.b64 da, {la, %4};\n"
         "mov.b64 db, {lb, %4};\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 pr, [%8], %9;\n"
         "tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, 1;\n"
 #endif
         "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%7];\n"
@@ -230,7 +233,6 @@ __device__ __forceinline__ bool umma_kblock_bf16_pair(uint32_t tmem_d, uint32_t 
         ".reg .pred pr, pa;\n"
         ".reg .b64 da, db;\n"
         ".reg .b32 la, lb;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 pr, [%8], %9;\n"
         "setp.ne.b32 pa, %6, 0;\n"
         "mov.b64 da, {%2, %4};\n"
         "mov.b64 db, {%3, %4};\n"
@@ -249,6 +251,7 @@ __device__ __forceinline__ bool umma_kblock_bf16_pair(uint32_t tmem_d, uint32_t 
         "add.u32 lb, %3, 6;\n"
         "mov.b64 da, {la, %4};\n"
         "mov.b64 db, {lb, %4};\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 pr, [%8], %9;\n"
         "tcgen05.mma.cta_group::2.kind::f16 [%1], da, db, %5, 1;\n"
         "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%7], %10;\n"
         "selp.b32 %0, 1, 0, pr;\n"
