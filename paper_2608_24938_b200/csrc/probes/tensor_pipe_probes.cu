@@ -143,7 +143,8 @@ static void run_mma(const char* name, int grid, int iters, int copies, int delay
 }
 
 // ---------------------------------------------------------------- pair: clusters of two CTAs, the leader's thread 0 issues
-// fused = 1: the library's one-sequence k-block (poll, 4 MMAs, commit) instead of separate instructions
+// FUSED 1 / 2: the library's one-sequence k-block (4 MMAs with a poll before the last, commit) instead of separate
+// instructions; 1 keeps this loop's own wait for the k-block issued four earlier (two barrier polls per k-block)
 template <int FUSED>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128, 1) pair_probe(int iters, ProbeOut* out) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -175,7 +176,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128, 1) pair_probe(i
         int bad = 0;
         for (int it = 0; it < iters && !bad; ++it) {
             const int slot = it & 3;
-            if (it >= 4 && !spin_wait(&bars[slot], ((it >> 2) - 1) & 1)) { bad = 1; break; }
+            // FUSED 2: the library sequence's own poll is the only barrier instruction of the loop, as in the kernel
+            if (FUSED != 2 && it >= 4 && !spin_wait(&bars[slot], ((it >> 2) - 1) & 1)) { bad = 1; break; }
             const uint32_t a_lo = a0 + (uint32_t)(it & 3) * (32768u >> 4);
             if (FUSED) {  // polls bars[4] (never arrived on: parity 1 reads as complete); the commit goes to both CTAs
                 ptx::umma_kblock_bf16_pair(tb, a_lo, a_lo + (16384u >> 4), (uint32_t)(hi >> 32), idesc, 1u, &bars[slot],
@@ -282,10 +284,12 @@ int main(int argc, char** argv) {
         const int smem = 4 * 32768 + 1024 + 64 * 1024;
         cudaFuncSetAttribute(pair_probe<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         cudaFuncSetAttribute(pair_probe<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        for (int fused : {0, 1})
+        cudaFuncSetAttribute(pair_probe<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        for (int fused : {0, 1, 2})
         for (int grid : {2, 148}) {
             for (int rep = 0; rep < 2; ++rep) {
-                if (fused) pair_probe<1><<<grid, 128, smem>>>(20000, d);
+                if (fused == 2) pair_probe<2><<<grid, 128, smem>>>(20000, d);
+                else if (fused == 1) pair_probe<1><<<grid, 128, smem>>>(20000, d);
                 else pair_probe<0><<<grid, 128, smem>>>(20000, d);
                 cudaError_t e = cudaDeviceSynchronize();
                 if (e != cudaSuccess) { printf("CUDA error %s\n", cudaGetErrorString(e)); return 1; }
@@ -295,7 +299,7 @@ int main(int argc, char** argv) {
             for (int i = 0; i < grid / 2; ++i) { cyc += h[i].cycles; ns += h[i].ns; bad += (int)h[i].err; }
             const double kb = cyc / (grid / 2) / 20000, ghz = cyc / ns;
             printf("%s SMs %3d: %6.1f cycles/k-block (%5.1f per M256 MMA), %.3f GHz, %6.1f ns/k-block%s\n",
-                   fused ? "library k-block sequence," : "separate instructions,   ", grid, kb, kb / 4, ghz, kb / ghz,
+                   fused == 2 ? "library k-block sequence, one poll per k-block, " : fused == 1 ? "library k-block sequence, two polls per k-block," : "separate instructions, one poll per k-block,    ", grid, kb, kb / 4, ghz, kb / ghz,
                    bad ? "  WAIT LIMIT HIT" : "");
         }
     }
