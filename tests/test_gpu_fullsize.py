@@ -15,8 +15,10 @@ def sample_tokens(T, n, seed=3):
     return np.sort(np.random.default_rng(seed).choice(T, size=min(n, T), replace=False)).astype(np.int64)
 
 
-def run_full(name, n_sample, decode_cases=None):
+def run_full(name, n_sample, decode_cases=None, prefill_tokens=None):
     cfg = si.CONFIGS[name]
+    if prefill_tokens:
+        cfg = si.scaled(cfg, prefill_tokens=prefill_tokens)
     case = Case(cfg, std=0.02)
     for Kp in cfg.k_pre:
         idx = sample_tokens(cfg.prefill_tokens, n_sample)
@@ -27,7 +29,7 @@ def run_full(name, n_sample, decode_cases=None):
         # properties that hold at any size: every token keeps K' distinct routed experts
         assert (np.diff(np.sort(got["ids"], 1), axis=1) > 0).all() if Kp > 1 else True
         assert np.array_equal(np.sort(got["perm"]), np.arange(cfg.prefill_tokens * Kp))
-    for M in (decode_cases or cfg.pool_m):
+    for M in (cfg.pool_m if decode_cases is None else decode_cases):
         got, ref = case.run_decode(M), case.oracle_decode(M)
         assert ref["min_gap"] > 1e-9, "degenerate input: tie at the pool boundary"
         check_decode_meta(got, ref, M)
@@ -37,6 +39,12 @@ def run_full(name, n_sample, decode_cases=None):
 
 def test_mixtral_shaped_full_size():
     run_full("mixtral", 48)
+
+
+def test_mixtral_shaped_long_prefill_runs_on_cta_pairs():
+    """16384 tokens = 128+ row tiles: both prefill GEMMs take the CTA-pair kernel with the odd last tiles on the
+    one-CTA kernel (the library's own choice, no override), K' = 1 so GEMM-2 writes y directly."""
+    run_full("mixtral", 48, decode_cases=(), prefill_tokens=16384)
 
 
 def test_qwen3_shaped_full_size():
