@@ -135,6 +135,27 @@ int exfold_calibrate(const exfold_layer *layer, const void *x_cal, const float *
                      void *cuda_stream);
 
 /*
+ * Calibration of several layers of one model in one call ("Calibration protocol": every MoE layer gets its own
+ * tables from the same calibration prompts). All jobs share the layer description (shape, dtype) and the options;
+ * each job names its own calibration inputs, expert weights and output tables (device pointers, as for
+ * exfold_calibrate). The jobs are enqueued back to back on the stream and the call synchronises once, at the end;
+ * tables are bit-identical to those of one exfold_calibrate call per job. `unobserved` (host, [n_jobs], may be NULL)
+ * receives each job's number of never-observed experts; the call returns EXFOLD_WARN_UNOBSERVED_EXPERT if any is
+ * positive. Workspace: exfold_workspace_bytes for the largest job (see exfold_calibrate). n_jobs <= EXFOLD_MAX_CALIB_JOBS.
+ */
+#define EXFOLD_MAX_CALIB_JOBS 256
+typedef struct {
+    const void *x_cal;        /* [m][d] */
+    const float *logits_cal;  /* [m][N] (mode 0) or NULL (mode 1) */
+    int64_t m;
+    const void *w_gate, *w_up, *w_down;
+    exfold_tables *out;
+} exfold_calib_job;
+int exfold_calibrate_layers(const exfold_layer *layer, const exfold_calib_job *jobs, int32_t n_jobs,
+                            const exfold_calib_opts *opts, int32_t *unobserved, void *ws, size_t ws_bytes,
+                            void *cuda_stream);
+
+/*
  * Prefill: token-level Top-K folding (Eq. 10, 12, 13, then Eq. 1 and 4 over the retained
  * routes only). x [T][d], logits [T][N] -> y [T][d]. k_pre = K' in [1, K]; k_pre = K is the
  * unfolded layer. Each token executes exactly K' routed experts (+ the shared expert).

@@ -30,7 +30,7 @@ EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibr
            "exfold_moe_decode", "exfold_moe_prefill_host", "exfold_moe_decode_host", "exfold_device_status",
            "exfold_status_string", "exfold_launch_count", "exfold_profile_enable", "exfold_profile_read",
            "exfold_moe_decode_noalloc", "exfold_static_pool_build", "exfold_moe_decode_static",
-           "exfold_moe_prefill_ex", "exfold_router_logits"]
+           "exfold_moe_prefill_ex", "exfold_router_logits", "exfold_calibrate_layers"]
 PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
                  "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
                  "simt_combine", "gemm1_pair_pass", "gemm2_pair_pass"]
@@ -48,6 +48,11 @@ class exfold_tables(C.Structure):
 class exfold_calib_opts(C.Structure):
     _fields_ = [("lambda_", C.c_float), ("clip_lo", C.c_float), ("clip_hi", C.c_float), ("eps", C.c_float),
                 ("mode", C.c_int32)]
+
+
+class exfold_calib_job(C.Structure):
+    _fields_ = [("x_cal", C.c_void_p), ("logits_cal", C.c_void_p), ("m", C.c_int64), ("w_gate", C.c_void_p),
+                ("w_up", C.c_void_p), ("w_down", C.c_void_p), ("out", C.POINTER(exfold_tables))]
 
 
 class exfold_prefill_meta(C.Structure):
@@ -81,6 +86,9 @@ def _load() -> C.CDLL:
     lib.exfold_calibrate.restype = C.c_int
     lib.exfold_calibrate.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_calib_opts),
                                      C.POINTER(exfold_tables), vp, sz, vp]
+    lib.exfold_calibrate_layers.restype = C.c_int
+    lib.exfold_calibrate_layers.argtypes = [C.POINTER(exfold_layer), C.POINTER(exfold_calib_job), i32,
+                                            C.POINTER(exfold_calib_opts), C.POINTER(C.c_int32), vp, sz, vp]
     for fn in (lib.exfold_moe_prefill, lib.exfold_moe_prefill_host):
         fn.restype = C.c_int
         fn.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables), i32, vp,
@@ -208,6 +216,21 @@ def exfold_calibrate(layer, x_cal, logits_cal, w_gate, w_up, w_down, out: exfold
     if rc < 0:
         raise ExfoldError(rc, "exfold_calibrate")
     return rc
+
+
+def exfold_calibrate_layers(layer, jobs, ws, lam=1e-3, clip_lo=-4.0, clip_hi=4.0, eps=1e-12, mode=0, stream=None):
+    """jobs: sequence of (x_cal, logits_cal, w_gate, w_up, w_down, out_tables). Returns (status, unobserved per job)."""
+    opts = exfold_calib_opts(lam, clip_lo, clip_hi, eps, mode)
+    arr = (exfold_calib_job * len(jobs))()
+    for j, (x_cal, logits_cal, w_gate, w_up, w_down, out) in enumerate(jobs):
+        arr[j] = exfold_calib_job(_ptr(x_cal), _ptr(logits_cal), x_cal.shape[0], _ptr(w_gate), _ptr(w_up),
+                                  _ptr(w_down), C.pointer(out))
+    un = (C.c_int32 * len(jobs))()
+    rc = lib.exfold_calibrate_layers(C.byref(layer), arr, len(jobs), C.byref(opts), un, _ptr(ws), ws.numel(),
+                                     _stream(stream))
+    if rc < 0:
+        raise ExfoldError(rc, "exfold_calibrate_layers")
+    return rc, list(un)
 
 
 def _prefill_meta(meta: Optional[dict]):

@@ -60,7 +60,7 @@ void prof_reset() {
 struct Plan {
     size_t status, ids, w, omit_src, omit_tgt, block_hist, offsets, work_start, totals, perm, row_tok, row_w,
         row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
-        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, work_ctr, total;
+        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, work_ctr, calib_warn, total;
 };
 
 bool valid_layer(const exfold_layer* l) {
@@ -87,6 +87,9 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
         return at;
     };
     p.status = take(sizeof(DeviceStatus));
+    // calibration: unobserved-expert count of each job of a call (ahead of everything whose size depends on the
+    // token count, so that jobs of different lengths share the slots)
+    p.calib_warn = take((size_t)EXFOLD_MAX_CALIB_JOBS * 4);
     p.ids = take(Rm * 4);
     p.w = take(Rm * 4);
     p.omit_src = take((size_t)Tm * l.top_k * 4);
@@ -564,9 +567,11 @@ int exfold_static_pool_build(const exfold_layer* layer, const exfold_tables* tab
     return EXFOLD_OK;
 }
 
-int exfold_calibrate(const exfold_layer* layer, const void* x_cal, const float* logits_cal, int64_t m,
-                     const void* w_gate, const void* w_up, const void* w_down, const exfold_calib_opts* opts,
-                     exfold_tables* out, void* ws, size_t ws_bytes, void* cuda_stream) {
+// Enqueues one calibration on the stream (no synchronisation); the number of unobserved experts lands in
+// warn_slot (device memory) when the stream gets there.
+static int calibrate_enqueue(const exfold_layer* layer, const void* x_cal, const float* logits_cal, int64_t m,
+                             const void* w_gate, const void* w_up, const void* w_down, const exfold_calib_opts* opts,
+                             exfold_tables* out, void* ws, size_t ws_bytes, void* cuda_stream, int job) {
     if (!valid_layer(layer) || !x_cal || !w_gate || !w_up || !w_down || !opts || !out || !ws)
         return EXFOLD_ERR_INVALID_ARG;
     if (!out->S || !out->L || !out->h || !out->lnh) return EXFOLD_ERR_INVALID_ARG;
@@ -669,10 +674,57 @@ int exfold_calibrate(const exfold_layer* layer, const void* x_cal, const float* 
     else
         EXFOLD_CUDA(launch_calib_stats(cs, s));
     EXFOLD_CUDA(launch_calib_finalize(cs, *opts, out->S, out->L, out->h, out->lnh, out->n_obs, unobs, s));
-    int un = 0;
-    EXFOLD_CUDA(cudaMemcpyAsync(&un, unobs, 4, cudaMemcpyDeviceToHost, s));
+    EXFOLD_CUDA(cudaMemcpyAsync(at<int32_t>(ws, pl.calib_warn) + job, unobs, 4, cudaMemcpyDeviceToDevice, s));
+    return EXFOLD_OK;
+}
+
+// The jobs' unobserved-expert counts, after the stream has drained
+static int calibrate_collect(const exfold_layer* layer, int64_t m_max, int Ke, int n_jobs, int32_t* warn, void* ws,
+                             cudaStream_t s) {
+    exfold_layer lc = *layer;
+    lc.n_shared = 0;
+    const Plan pl = make_plan(lc, m_max, Ke);
+    int32_t un[EXFOLD_MAX_CALIB_JOBS];
+    EXFOLD_CUDA(cudaMemcpyAsync(un, at<int32_t>(ws, pl.calib_warn), (size_t)n_jobs * 4, cudaMemcpyDeviceToHost, s));
     EXFOLD_CUDA(cudaStreamSynchronize(s));
-    return un > 0 ? EXFOLD_WARN_UNOBSERVED_EXPERT : EXFOLD_OK;
+    int any = 0;
+    for (int j = 0; j < n_jobs; ++j) {
+        if (warn) warn[j] = un[j];
+        any |= un[j] > 0;
+    }
+    return any ? EXFOLD_WARN_UNOBSERVED_EXPERT : EXFOLD_OK;
+}
+
+int exfold_calibrate(const exfold_layer* layer, const void* x_cal, const float* logits_cal, int64_t m,
+                     const void* w_gate, const void* w_up, const void* w_down, const exfold_calib_opts* opts,
+                     exfold_tables* out, void* ws, size_t ws_bytes, void* cuda_stream) {
+    int rc = calibrate_enqueue(layer, x_cal, logits_cal, m, w_gate, w_up, w_down, opts, out, ws, ws_bytes, cuda_stream, 0);
+    if (rc != EXFOLD_OK) return rc;
+    return calibrate_collect(layer, m, opts->mode == 1 ? layer->n_experts : layer->top_k, 1, nullptr, ws,
+                             reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int exfold_calibrate_layers(const exfold_layer* layer, const exfold_calib_job* jobs, int32_t n_jobs,
+                            const exfold_calib_opts* opts, int32_t* unobserved, void* ws, size_t ws_bytes,
+                            void* cuda_stream) {
+    if (!valid_layer(layer) || !jobs || !opts || n_jobs < 1 || n_jobs > EXFOLD_MAX_CALIB_JOBS) return EXFOLD_ERR_INVALID_ARG;
+    if (opts->mode != 0 && opts->mode != 1) return EXFOLD_ERR_INVALID_ARG;
+    int64_t m_max = 0;
+    for (int j = 0; j < n_jobs; ++j) {
+        if (!jobs[j].out || jobs[j].m < 1) return EXFOLD_ERR_INVALID_ARG;
+        m_max = std::max<int64_t>(m_max, jobs[j].m);
+    }
+    // Every job uses the plan of the largest one, so that the jobs' warning slots sit at one place; the jobs run
+    // one after the other on the stream and share the rest of the workspace.
+    const int Ke = opts->mode == 1 ? layer->n_experts : layer->top_k;
+    if (ws_bytes < exfold_workspace_bytes(layer, m_max, Ke)) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
+    for (int j = 0; j < n_jobs; ++j) {
+        const exfold_calib_job& b = jobs[j];
+        int rc = calibrate_enqueue(layer, b.x_cal, b.logits_cal, b.m, b.w_gate, b.w_up, b.w_down, opts, b.out, ws,
+                                   ws_bytes, cuda_stream, j);
+        if (rc != EXFOLD_OK) return rc;
+    }
+    return calibrate_collect(layer, m_max, Ke, n_jobs, unobserved, ws, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
 int exfold_router_logits(const exfold_layer* layer, const void* x, const void* w_router, int64_t T, float* logits,

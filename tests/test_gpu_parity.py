@@ -73,6 +73,42 @@ def test_calibrate_matches_oracle(mode):
     assert (np.diag(S.cpu().numpy()) == 1).all() and (np.diag(L.cpu().numpy()) == 0).all()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_calibrate_layers_equals_one_call_per_layer(dtype):
+    """Three layers (own weights, calibration sets of different lengths) in one call: tables bit-identical to
+    those of three exfold_calibrate calls, per-job unobserved counts as returned by the single calls."""
+    cfg = TINY if dtype == "f32" else small_bf16(n_experts=8, top_k=2, hidden=128, inter=192, calib_tokens=300)
+    cases = [Case(si.scaled(cfg, seed=cfg.seed + j), std=0.02, correlated=0.5) for j in range(3)]
+    ex, dev = cases[0].ex, cases[0].dev
+    N, K = cfg.n_experts, cfg.top_k
+    ms = [cfg.calib_tokens, cfg.calib_tokens // 2 + 3, 40]
+
+    def fresh():
+        S = torch.full((N, N), float("nan"), device=dev)
+        return dict(S=S, L=torch.full_like(S, float("nan")), h=torch.full((N,), float("nan"), device=dev),
+                    lnh=torch.empty(N, device=dev), n_obs=torch.full((N, N), -1, dtype=torch.int32, device=dev))
+
+    inputs = [(si.hidden_states(c.cfg, m, "x_cal").to(dev), si.router_logits(c.cfg, m, "logits_cal").to(dev))
+              for c, m in zip(cases, ms)]
+    ws = ex.alloc_workspace(cases[0].layer, max(ms), K)
+    single, rcs = [], []
+    for c, (xc, lc) in zip(cases, inputs):
+        t = fresh()
+        rcs.append(ex.exfold_calibrate(c.layer, xc, lc, c.d_wg, c.d_wu, c.d_wd,
+                                       ex.make_tables(t["S"], t["L"], t["h"], t["lnh"], t["n_obs"]), ws))
+        single.append({k: v.cpu().numpy() for k, v in t.items()})
+    batched = [fresh() for _ in cases]
+    tabs = [ex.make_tables(t["S"], t["L"], t["h"], t["lnh"], t["n_obs"]) for t in batched]
+    ws.fill_(0xFF)
+    rc, unobserved = ex.exfold_calibrate_layers(
+        cases[0].layer, [(xc, lc, c.d_wg, c.d_wu, c.d_wd, tab) for c, (xc, lc), tab in zip(cases, inputs, tabs)], ws)
+    assert rc == max(rcs)
+    assert [int(u > 0) for u in unobserved] == rcs
+    for a, b in zip(single, batched):
+        for k in a:
+            assert np.array_equal(a[k], b[k].cpu().numpy(), equal_nan=True), k
+
+
 def test_calibrate_common_input_many_experts_fp32():
     """Common-input mode with N >= 32 takes the Gram-product form of the pair sums; fp32 layer, tight bound."""
     cfg = si.LayerConfig("f32_many", 40, 0, 96, 64, 2, "f32", 64, (1,), 16, (4,))

@@ -83,6 +83,19 @@ def test_bad_arguments_are_rejected_before_launch(ex):
     rc = ex.lib.exfold_calibrate(C.byref(layer), p, p, 16, p, p, p, C.byref(opts), C.byref(out), p, big, None)
     assert rc == ex.EXFOLD_ERR_INVALID_ARG                     # unknown calibration mode
     assert ex.lib.exfold_device_status(None, None) == ex.EXFOLD_ERR_INVALID_ARG
+    good = ex.exfold_calib_opts(1e-3, -4, 4, 1e-12, 0)
+    jobs = (ex.exfold_calib_job * 2)(ex.exfold_calib_job(p, p, 16, p, p, p, C.pointer(out)),
+                                     ex.exfold_calib_job(p, p, 16, p, p, p, C.pointer(out)))
+
+    def layers(jobs=jobs, n=2, opts=good, wsb=big):
+        return ex.lib.exfold_calibrate_layers(C.byref(layer), jobs, n, C.byref(opts), None, p, wsb, None)
+
+    assert layers(n=0) == ex.EXFOLD_ERR_INVALID_ARG
+    assert layers(n=257) == ex.EXFOLD_ERR_INVALID_ARG            # more jobs than EXFOLD_MAX_CALIB_JOBS
+    assert layers(opts=opts) == ex.EXFOLD_ERR_INVALID_ARG        # unknown calibration mode
+    assert layers(wsb=1024) == ex.EXFOLD_ERR_WORKSPACE_TOO_SMALL
+    bad = (ex.exfold_calib_job * 1)(ex.exfold_calib_job(p, p, 0, p, p, p, C.pointer(out)))
+    assert layers(jobs=bad, n=1) == ex.EXFOLD_ERR_INVALID_ARG    # a job without tokens
 
     def router(layer=layer, x=p, wr=p, T=4, lg=p, ws=p, wsb=big):
         return ex.lib.exfold_router_logits(C.byref(layer), x, wr, T, lg, ws, wsb, None)
