@@ -60,7 +60,7 @@ void prof_reset() {
 struct Plan {
     size_t status, ids, w, omit_src, omit_tgt, block_hist, offsets, work_start, totals, perm, row_tok, row_w,
         row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
-        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, work_ctr, calib_warn, total;
+        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, calib_warn, total;
 };
 
 bool valid_layer(const exfold_layer* l) {
@@ -98,7 +98,6 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
     p.offsets = take((G + 2) * 4);
     p.work_start = take((G + 2) * 4);
     p.totals = take(16);
-    p.work_ctr = take(16);
     p.perm = take(Rm * 4);
     p.inv_pos = take(Rm * 4);
     p.row_tok = take(Rtot * 4);
@@ -370,7 +369,6 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
     cp.row_w = at<float>(ws, pl.row_w); cp.row_exp = at<int32_t>(ws, pl.row_exp);
     cp.inv_pos = at<int32_t>(ws, pl.inv_pos);
-    cp.work_ctr = at<int32_t>(ws, pl.work_ctr);
     { ProfScope ps(2, s); EXFOLD_CUDA(launch_prefill_scatter(cp, s)); }
 
     if (bf16) {
@@ -388,12 +386,10 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             if (pairs1) {
                 { ProfScope pp(12, s); EXFOLD_CUDA(launch_grouped_gemm1_pair(g, grid1, s)); }
                 g.odd_only = 1;
-                g.work_ctr = cp.work_ctr;
                 grid1 = (int)std::min<int64_t>(sm_count(), (int64_t)G * g.n_ntiles);
             }
             EXFOLD_CUDA(launch_grouped_gemm1(g, grid1, s));
             g.odd_only = 0;
-            g.work_ctr = nullptr;
         }
         g.tm_a = tm_h; g.tm_b0 = tm_wd; g.tm_b1 = tm_wd_half; g.n_ntiles = (d + 255) / 256;
         // K' = 1 without a shared expert: every token is written once, straight into y. Otherwise each
@@ -407,12 +403,10 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             if (pairs2) {
                 { ProfScope pp(13, s); EXFOLD_CUDA(launch_grouped_gemm2_pair(g, grid2, s)); }
                 g.odd_only = 1;
-                g.work_ctr = cp.work_ctr + 1;
                 grid2 = (int)std::min<int64_t>(sm_count(), (int64_t)G * g.n_ntiles);
             }
             EXFOLD_CUDA(launch_grouped_gemm2(g, grid2, s));
             g.odd_only = 0;
-            g.work_ctr = nullptr;
         }
         if (!direct) {
             ProfScope ps(5, s);

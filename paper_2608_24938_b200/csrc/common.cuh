@@ -156,7 +156,6 @@ struct PrefillScatterParams {
     float* row_w;       // [R + T*n_shared]
     int32_t* row_exp;   // [R + T*n_shared]
     int32_t* inv_pos;   // [R] sorted row of each route (inverse of perm); may be null
-    int32_t* work_ctr;  // [2] cleared here: work-item counters of the GEMMs that follow (may be null)
 };
 
 cudaError_t launch_prefill_route(const PrefillRouteParams& p, cudaStream_t s);
@@ -274,7 +273,6 @@ struct GroupedGemmParams {
     float* o32;                 // GEMM-2, calibration: unweighted fp32 outputs O32[row][d] (null: the epilogues above)
     int x_rows;                 // GEMM-1: rows of x; a group that reads x directly starts at row (row0 - R) % x_rows
     int odd_only;               // 1: only each group's last row tile, and only if its tile count is odd (the rest ran on CTA pairs)
-    int* work_ctr;              // prefill: zeroed counter from which the CTAs draw their work items (null: item = CTA index + k * grid)
     DeviceStatus* status;
 };
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s);

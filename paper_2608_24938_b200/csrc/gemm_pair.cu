@@ -104,10 +104,6 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
         ptx::tmem_relinquish_pair();
     }
     grid_dep_wait();  // everything below reads what the routing kernels (or GEMM-1) wrote
-    // The next launch is always the odd-tile pass of the same GEMM: it depends on nothing this kernel writes, cannot
-    // share an SM with a CTA of this kernel (shared memory), and waits for this grid only at its very end. Released
-    // here, its CTAs take over the SMs one by one as the pairs run out of work, instead of after the last pair.
-    if (threadIdx.x == 0) grid_dep_launch();
     const int G = p.G;
     for (int i = threadIdx.x; i <= G; i += kPThreads) s_off[i] = p.offsets[i];
     ptx::tc_fence_before();
@@ -329,6 +325,7 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
     }
 
     // ------------------------------------------------ teardown
+    if (threadIdx.x == 64) grid_dep_launch();  // after the epilogue loop, as in the one-CTA kernel
     ptx::tc_fence_before();
     __syncthreads();
     if (abort_s) __nanosleep(100000);  // let any copy still in flight land before shared memory is released

@@ -84,60 +84,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Work items of one CTA, in the order it takes them. Static: item w_begin + pos * w_stride. Dynamic (work_ctr != null,
-// the odd-tile pass): the first producer thread draws the next item from a global counter - one item ahead, so the
-// round trip overlaps the loads of the current one - and publishes it in a shared ring; the other roles read the
-// ring. CTAs that start early or run fast simply draw more items. Every role calls next() once per position.
-constexpr int kItemRing = 32;  // > the positions any two roles of a CTA can be apart (ring stages + accumulators)
-struct ItemSeq {
-    int w_begin, w_stride, total;
-    int* ctr;                    // null: static
-    volatile int* ring;          // shared: [kItemRing]
-    volatile int* published;     // shared: number of ring entries written
-    // the drawing thread: returns item `pos` (or -1) and draws + publishes item pos + 1 ahead of time
-    __device__ __forceinline__ int draw(int pos, int& ahead) {
-        if (ctr == nullptr) {
-            const int w = w_begin + pos * w_stride;
-            return w < total ? w : -1;
-        }
-        if (pos == 0) {
-            ahead = atomicAdd(ctr, 1);
-            ring[0] = ahead;
-            __threadfence_block();
-            *published = 1;
-        }
-        const int w = ahead;
-        if (w >= total) return -1;
-        ahead = atomicAdd(ctr, 1);
-        ring[(pos + 1) % kItemRing] = ahead;
-        __threadfence_block();
-        *published = pos + 2;
-        return w;
-    }
-    // every other role: item `pos` (or -1), or -2 if the ring entry never appeared
-    __device__ __forceinline__ int next(int pos, volatile int* abort_flag, DeviceStatus* st) {
-        if (ctr == nullptr) {
-            const int w = w_begin + pos * w_stride;
-            return w < total ? w : -1;
-        }
-        uint64_t t0 = 0;
-        for (uint32_t it = 0; *published <= pos; ++it) {
-            if ((it & 255u) == 255u) {
-                if (*abort_flag || ((volatile int*)&st->code)[0] != 0) return -2;
-                const uint64_t now = ptx::globaltimer_ns();
-                if (t0 == 0) t0 = now;
-                else if (now - t0 > ptx::kWaitLimitNs) {
-                    *abort_flag = 1;
-                    report_timeout(st, 5);
-                    return -2;
-                }
-            }
-        }
-        const int w = ring[pos % kItemRing];
-        return w < total ? w : -1;
-    }
-};
-
 // MODE 0: gate/up + SwiGLU -> H; MODE 1: down + weighted scatter -> y.
 // DEC (decode) adds what only the expert-pool path needs: a group -> expert map, a group count that is
 // known only on the device, and split-K for GEMM-2. The prefill instantiations compile all of it away.
@@ -153,8 +99,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     __shared__ int s_off[kMaxGroups + 1];
     __shared__ int s_ws[kMaxGroups + 1];
     __shared__ int s_exp[kMaxGroups + 1];
-    __shared__ int s_item[kItemRing];
-    __shared__ int s_item_n;
 
     unsigned char* tiles =
         reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -182,17 +126,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
             ptx::mbar_init(&tempty_bar[s], 4);
         }
         abort_s = 0;
-        s_item_n = 0;
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
         ptx::tmem_alloc(&tmem_base_s, kTmemCols);
         ptx::tmem_relinquish();
     }
-    // The odd-tile pass (odd_only) follows the CTA-pair pass of the same GEMM, which released it only after all of
-    // its own CTAs had seen their inputs complete: the inputs of this pass are complete too, and it waits for the
-    // pair pass at its end instead (so that whoever waits for this grid also has the pair pass's results).
-    if (DEC || !p.odd_only) grid_dep_wait();  // everything below reads what the routing kernels (or GEMM-1) wrote
+    grid_dep_wait();  // everything below reads what the routing kernels (or GEMM-1) wrote
     int G = p.G;
     if (DEC) {  // the number of groups (pool size) is known only on the device
         const int gd = *p.n_groups_dev;
@@ -239,7 +179,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     const int eff_grid = rounds > 0 ? (total + rounds - 1) / rounds : 0;
     const int w_begin = (int)blockIdx.x < eff_grid ? (int)blockIdx.x : total;  // idle CTAs see no work
     const int w_stride = eff_grid > 0 ? eff_grid : 1;
-    ItemSeq seq{w_begin, w_stride, total, DEC ? nullptr : p.work_ctr, s_item, &s_item_n};
     const int nkb = (MODE == 0 ? p.d : p.I) / kBK;
     const int kb_per = (nkb + ks - 1) / ks;
     // Stage geometry. Prefill: 16 KB A + 32 KB B, 4 stages (compile-time). Decode: the A box has only
@@ -257,10 +196,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
             const int me = warp == 0 ? 0 : warp - 5;
             int stage = 0, phase = 0, turn = 0;
             bool ok = true;
-            int ahead = 0;
-            for (int pos = 0; ok; ++pos) {
-                const int w = me == 0 ? seq.draw(pos, ahead) : seq.next(pos, abort_flag, p.status);
-                if (w < 0) break;
+            for (int w = w_begin; w < total && ok; w += w_stride) {
                 const WorkItem it = decode_work(w, G, nt, ks, s_off, s_ws, DEC ? 0 : p.odd_only);
                 const int kb0 = it.kpart * kb_per, kb1 = min(nkb, kb0 + kb_per);
                 // per-tile constants stay in registers: the k-loop below is the latency-critical path
@@ -316,9 +252,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
             uint32_t a_lo = lo0;
             bool ok = true;
             bool ready = false;
-            for (;ok; ++iter) {
-                const int w = seq.next(iter, abort_flag, p.status);
-                if (w < 0) break;
+            for (int w = w_begin; w < total && ok; w += w_stride, ++iter) {
                 const int as = iter & 1, aphase = (iter >> 1) & 1;
                 bool got;
                 EXFOLD_TRACE_ADD(tr_wait2, got = ptx::mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag, p.status, 2));
@@ -372,11 +306,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         // ------------------------------------------------ epilogue warps (TMEM lane quadrant = warp % 4)
         const int q = warp & 3;
         int iter = 0;
-        for (;; ++iter) {
-            int w = 0;
-            if (lane == 0) w = seq.next(iter, abort_flag, p.status);
-            w = __shfl_sync(0xffffffffu, w, 0);
-            if (w < 0) break;
+        for (int w = w_begin; w < total; w += w_stride, ++iter) {
             const int as = iter & 1, aphase = (iter >> 1) & 1;
             const WorkItem it = decode_work(w, G, nt, ks, s_off, s_ws, DEC ? 0 : p.odd_only);
             // lane 0 waits; the warp takes one decision, so the warp-wide TMEM loads below stay convergent
@@ -480,7 +410,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         EXFOLD_TRACE_SET(kTr, 8, tr_wait);
         EXFOLD_TRACE_SET(kTr, 11, ptx::globaltimer_ns());
     }
-    if (!DEC && p.odd_only) grid_dep_wait();
     ptx::tc_fence_before();
     __syncthreads();
     if (abort_s) __nanosleep(100000);  // let any copy still in flight land before shared memory is released

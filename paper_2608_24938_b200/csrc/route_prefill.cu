@@ -204,7 +204,6 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_scatter_kernel(PrefillS
         cnt[e] = off + part_pre[0][e] + part_pre[1][e] + part_pre[2][e] + part_pre[3][e];
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {  // group offsets and the row-tile prefix for the GEMM work list
-        if (p.work_ctr != nullptr) p.work_ctr[0] = p.work_ctr[1] = 0;  // the GEMMs' odd-tile passes draw their items from these
         const int G = N + p.n_shared;
         int off = 0, tiles = 0;
         for (int g = 0; g < G; ++g) {
