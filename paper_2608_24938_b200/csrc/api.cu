@@ -183,6 +183,24 @@ int pair_gemm_mode() {
     return mode < 0 || mode > 2 ? 1 : mode;
 }
 
+// Second stream (and fork / join events) on which the odd-tile passes of a prefill call run beside the CTA-pair
+// passes. Created once per host thread, on first use, and kept for the life of the process.
+struct SideStream {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr, mid = nullptr;
+    bool ok = false;
+};
+SideStream& side_stream() {
+    static thread_local SideStream h;
+    if (!h.ok) {
+        h.ok = cudaStreamCreateWithFlags(&h.stream, cudaStreamNonBlocking) == cudaSuccess &&
+               cudaEventCreateWithFlags(&h.fork, cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventCreateWithFlags(&h.join, cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventCreateWithFlags(&h.mid, cudaEventDisableTiming) == cudaSuccess;
+    }
+    return h;
+}
+
 int sm_count() {
     static int n = 0;
     if (!n) {
@@ -321,21 +339,15 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     const bool direct = bf16 && Kp == 1 && l.n_shared == 0;  // every token is written exactly once
 
     CUtensorMap tm_xs, tm_x, tm_wg, tm_wu, tm_h, tm_wd, tm_wd_half;
-    // A GEMM with enough work runs every group's row tiles two at a time on CTA pairs (gemm_pair.cu: a third less
-    // operand traffic per SM, a deeper ring, the tensor pipe busy > 95 % of the main loop) and leaves only a group's
-    // odd last tile to the one-CTA kernel. The pair pass pays when the call is large (>= 48 row tiles), few tiles
-    // are odd ones (about one per two groups; at most one tile in eight) and the pair items fill the 74 CTA pairs
-    // for several rounds; otherwise the one-CTA kernel alone is as fast or faster (measured against it: Mixtral shape,
-    // 4096 tokens = 36 tiles: +0.4 %; Qwen3 shape, one tile in five odd: +4 to +8 %; Mixtral shape 6144 / 8192 /
-    // 16384 / 32768 tokens: -2 / -8 / -13 / -16 %; GLM shape: -6 %).
+    // A call with enough work (>= 24 row tiles of 128 sorted rows) runs every group's row tiles two at a time on CTA
+    // pairs (gemm_pair.cu: a third less operand traffic per SM, a deeper ring, the tensor pipe busy > 95 % of the
+    // main loop) and only a group's odd last tile on the one-CTA kernel, the two passes side by side (below).
+    // Measured against the one-CTA kernel alone: Mixtral shape 4096 / 8192 / 16384 / 32768 tokens -3 / -9 / -14 /
+    // -16 %, GLM shape -8 %, Qwen3 shape (half of the experts own a single tile) -1 %.
     const int64_t tiles_est = Rtot / kTileM + G / 2;
-    const int64_t pair_est = std::max<int64_t>(0, (tiles_est - G / 2) / 2);
     const int mode = pair_gemm_mode();
-    const bool pairs_ok = bf16 && kGemmBK == 64 && mode == 1 && tiles_est >= 48 && (int64_t)(G / 2) * 8 <= tiles_est;
-    const bool pairs_all = bf16 && kGemmBK == 64 && mode == 2 && Rtot >= 2 * kTileM;
-    const int n_pairs_hw = std::max(1, sm_count() / 2);
-    const bool pairs1 = pairs_all || (pairs_ok && pair_est * ((I + 127) / 128) >= 6 * (int64_t)n_pairs_hw);
-    const bool pairs2 = pairs_all || (pairs_ok && pair_est * ((d + 255) / 256) >= 6 * (int64_t)n_pairs_hw);
+    const bool pairs = bf16 && kGemmBK == 64 && (mode == 2 ? Rtot >= 2 * kTileM : mode == 1 && tiles_est >= 24);
+    const int sms = sm_count() & ~1;
     if (bf16) {
         const uint64_t E = (uint64_t)G;
         bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)R, d, 128) && make_tmap(&tm_x, x, (uint64_t)T, d, 128) &&
@@ -380,33 +392,47 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
         g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = cp.row_tok; g.row_w = cp.row_w;
         g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
         const int64_t max_tiles = Rtot / kTileM + G;
-        int grid1 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
-        {
-            ProfScope ps(3, s);
-            if (pairs1) {
-                { ProfScope pp(12, s); EXFOLD_CUDA(launch_grouped_gemm1_pair(g, grid1, s)); }
-                g.odd_only = 1;
-                grid1 = (int)std::min<int64_t>(sm_count(), (int64_t)G * g.n_ntiles);
-            }
-            EXFOLD_CUDA(launch_grouped_gemm1(g, grid1, s));
-            g.odd_only = 0;
-        }
-        g.tm_a = tm_h; g.tm_b0 = tm_wd; g.tm_b1 = tm_wd_half; g.n_ntiles = (d + 255) / 256;
+        const int nt1 = (I + 127) / 128, nt2 = (d + 255) / 256;
+        GroupedGemmParams g2 = g;  // GEMM-2: H x W_down -> y (or the per-route buffer O)
+        g2.tm_a = tm_h; g2.tm_b0 = tm_wd; g2.tm_b1 = tm_wd_half; g2.n_ntiles = nt2;
         // K' = 1 without a shared expert: every token is written once, straight into y. Otherwise each
         // route's weighted output goes to O (bf16, sorted rows) and the combine kernel sums per token.
-        g.y32 = nullptr;
-        g.y = direct ? reinterpret_cast<__nv_bfloat16*>(y) : at<__nv_bfloat16>(ws, pl.obuf);
-        g.store_rows = direct ? 0 : 1;
-        int grid2 = (int)std::min<int64_t>(sm_count(), max_tiles * g.n_ntiles);
-        {
-            ProfScope ps(4, s);
-            if (pairs2) {
-                { ProfScope pp(13, s); EXFOLD_CUDA(launch_grouped_gemm2_pair(g, grid2, s)); }
-                g.odd_only = 1;
-                grid2 = (int)std::min<int64_t>(sm_count(), (int64_t)G * g.n_ntiles);
+        g2.y = direct ? reinterpret_cast<__nv_bfloat16*>(y) : at<__nv_bfloat16>(ws, pl.obuf);
+        g2.store_rows = direct ? 0 : 1;
+        if (!pairs) {
+            { ProfScope ps(3, s); EXFOLD_CUDA(launch_grouped_gemm1(g, (int)std::min<int64_t>(sm_count(), max_tiles * nt1), s)); }
+            { ProfScope ps(4, s); EXFOLD_CUDA(launch_grouped_gemm2(g2, (int)std::min<int64_t>(sm_count(), max_tiles * nt2), s)); }
+        } else {
+            // Both passes are launched over all SMs, the pair pass on the caller's stream and the odd-tile pass on a
+            // second one; on the device each keeps its share of the SM pairs (pair_pass_clusters of the actual tile
+            // counts) and its other CTAs leave at once, so the two grids settle side by side whatever the routing.
+            // Rows of whole tile pairs and rows of odd last tiles never meet before the combine step, so each pass
+            // of GEMM-2 follows the same pass of GEMM-1 on its own stream: caller's stream: GEMM-1 pairs -> GEMM-2
+            // pairs; side stream: GEMM-1 odd tiles -> GEMM-2 odd tiles; joined before the combine kernel (or the
+            // end of the call). With per-kernel timing on, the streams also join between the two GEMMs.
+            SideStream& side = side_stream();
+            if (!side.ok) return EXFOLD_ERR_CUDA;
+            GroupedGemmParams go1 = g, go2 = g2;
+            go1.odd_only = go2.odd_only = 1;
+            g.side_by_side = g2.side_by_side = go1.side_by_side = go2.side_by_side = 1;
+            EXFOLD_CUDA(cudaEventRecord(side.fork, s));
+            EXFOLD_CUDA(cudaStreamWaitEvent(side.stream, side.fork, 0));
+            {
+                ProfScope ps(3, s);
+                { ProfScope pp(12, s); EXFOLD_CUDA(launch_grouped_gemm1_pair(g, sms, s)); }
+                EXFOLD_CUDA(launch_grouped_gemm1_odd(go1, sms, side.stream));
+                if (g_prof.on) {
+                    EXFOLD_CUDA(cudaEventRecord(side.mid, side.stream));
+                    EXFOLD_CUDA(cudaStreamWaitEvent(s, side.mid, 0));
+                }
             }
-            EXFOLD_CUDA(launch_grouped_gemm2(g, grid2, s));
-            g.odd_only = 0;
+            {
+                ProfScope ps(4, s);
+                { ProfScope pp(13, s); EXFOLD_CUDA(launch_grouped_gemm2_pair(g2, sms, s)); }
+                EXFOLD_CUDA(launch_grouped_gemm2_odd(go2, sms, side.stream));
+                EXFOLD_CUDA(cudaEventRecord(side.join, side.stream));
+                EXFOLD_CUDA(cudaStreamWaitEvent(s, side.join, 0));
+            }
         }
         if (!direct) {
             ProfScope ps(5, s);

@@ -273,13 +273,41 @@ struct GroupedGemmParams {
     float* o32;                 // GEMM-2, calibration: unweighted fp32 outputs O32[row][d] (null: the epilogues above)
     int x_rows;                 // GEMM-1: rows of x; a group that reads x directly starts at row (row0 - R) % x_rows
     int odd_only;               // 1: only each group's last row tile, and only if its tile count is odd (the rest ran on CTA pairs)
+    int side_by_side;           // 1: the CTA-pair pass and the odd-tile pass run at the same time (two streams), both
+                                //    launched over all SMs; each keeps its share of SM pairs (pair_pass_clusters) and
+                                //    the CTAs beyond it leave at once
     DeviceStatus* status;
 };
+// SM pairs, of n_clusters, that the CTA-pair pass keeps when the odd-tile pass runs beside it on the other
+// 2 * (n_clusters - P) SMs. Both kernels evaluate this on the device from the same group offsets, so they agree.
+// Side by side, a pair item takes a cluster ~0.73 of the time an odd item takes one SM (measured on the Mixtral shape:
+// 25.9 against 35.7 us per 64-k-block item; the one-CTA kernel is the hungrier of the two for L2 bandwidth and slows
+// down more beside the other); the choice minimises the longer of the two passes, counted in rounds of items.
+__host__ __device__ inline int pair_pass_clusters(int pair_items, int odd_items, int n_clusters) {
+    if (odd_items <= 0) return n_clusters;
+    if (pair_items <= 0) return 0;
+    int best = 1;
+    float best_t = 3.0e38f;
+    for (int P = 1; P < n_clusters; ++P) {
+        const int Q = 2 * (n_clusters - P);
+        const float tp = 0.73f * (float)((pair_items + P - 1) / P), to = (float)((odd_items + Q - 1) / Q);
+        const float t = tp > to ? tp : to;
+        if (t < best_t) {
+            best_t = t;
+            best = P;
+        }
+    }
+    return best;
+}
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s);
 cudaError_t launch_grouped_gemm2(const GroupedGemmParams& p, int grid, cudaStream_t s);
 // Prefill on CTA pairs: every group's row tiles two at a time (a last odd tile is left to the kernels above with
 // odd_only = 1). GEMM-2 needs tm_b1 = W_down with 128-row boxes. No grp_expert, no K split, y32 = null, o32 = null.
 cudaError_t launch_grouped_gemm1_pair(const GroupedGemmParams& p, int grid, cudaStream_t s);
 cudaError_t launch_grouped_gemm2_pair(const GroupedGemmParams& p, int grid, cudaStream_t s);
+// The odd-tile pass beside them (p.odd_only = 1; prefill instantiation), launched two CTAs at a time so that the two
+// grids share the GPU by whole SM pairs
+cudaError_t launch_grouped_gemm1_odd(const GroupedGemmParams& p, int grid, cudaStream_t s);
+cudaError_t launch_grouped_gemm2_odd(const GroupedGemmParams& p, int grid, cudaStream_t s);
 
 }  // namespace exfold

@@ -76,12 +76,13 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
     __shared__ int abort_s;
     __shared__ int s_off[kMaxGroups + 1];
     __shared__ int s_wp[kMaxGroups + 1];
+    __shared__ int s_n_odd;  // groups with an odd number of row tiles
 
     unsigned char* tiles =
         reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = (int)ptx::cluster_ctarank();  // 0 = leader
-    const int pair_id = (int)blockIdx.x >> 1, n_pairs = (int)gridDim.x >> 1;
+    const int pair_id = (int)blockIdx.x >> 1, n_launched = (int)gridDim.x >> 1;
     // GEMM-1: the leader stages W_gate rows, its peer W_up rows; GEMM-2: both halves come from W_down (tm_b1: 128-row box)
     const CUtensorMap* tma_b = MODE == 0 ? (rank == 0 ? &p.tm_b0 : &p.tm_b1) : &p.tm_b1;
     if (threadIdx.x == 0) {
@@ -104,16 +105,23 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
         ptx::tmem_relinquish_pair();
     }
     grid_dep_wait();  // everything below reads what the routing kernels (or GEMM-1) wrote
+#ifdef EXFOLD_TRACE_OVERLAP
+    if (threadIdx.x == 0 && MODE == 0) g_trace[2][blockIdx.x][0] = ptx::globaltimer_ns();
+#endif
     const int G = p.G;
     for (int i = threadIdx.x; i <= G; i += kPThreads) s_off[i] = p.offsets[i];
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 0) {  // prefix of whole row-tile pairs per group, 32 groups per step
-        int carry = 0;
+        int carry = 0, odd = 0;
         for (int g0 = 0; g0 < G; g0 += 32) {
             const int g = g0 + lane;
             int pairs = 0;
-            if (g < G) pairs = ((s_off[g + 1] - s_off[g] + kTileM - 1) / kTileM) >> 1;
+            if (g < G) {
+                const int tiles = (s_off[g + 1] - s_off[g] + kTileM - 1) / kTileM;
+                pairs = tiles >> 1;
+                odd += tiles & 1;
+            }
             int incl = pairs;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -123,7 +131,11 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
             if (g < G) s_wp[g] = carry + incl - pairs;
             carry += __shfl_sync(0xffffffffu, incl, 31);
         }
-        if (lane == 0) s_wp[G] = carry;
+        odd = __reduce_add_sync(0xffffffffu, odd);
+        if (lane == 0) {
+            s_wp[G] = carry;
+            s_n_odd = odd;
+        }
     }
     __syncthreads();
     ptx::cluster_sync_all();  // both CTAs' barriers are initialised and their tensor memory allocated
@@ -131,7 +143,9 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
     const uint32_t tmem_base = tmem_base_s;
     const int nt = p.n_ntiles;
     const int total = s_wp[G] * nt;
-    const int rounds = (total + n_pairs - 1) / n_pairs;
+    // beside the odd-tile pass this pass keeps only its share of the SM pairs; the other clusters leave at once
+    const int n_pairs = p.side_by_side ? pair_pass_clusters(total, s_n_odd * nt, n_launched) : n_launched;
+    const int rounds = n_pairs > 0 ? (total + n_pairs - 1) / n_pairs : 0;
     const int eff = rounds > 0 ? (total + rounds - 1) / rounds : 0;  // pairs that take work and finish together
     const int w_begin = pair_id < eff ? pair_id : total;
     const int w_stride = eff > 0 ? eff : 1;
@@ -325,6 +339,9 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
     }
 
     // ------------------------------------------------ teardown
+#ifdef EXFOLD_TRACE_OVERLAP
+    if (threadIdx.x == 0 && MODE == 0) g_trace[2][blockIdx.x][1] = ptx::globaltimer_ns();
+#endif
     if (threadIdx.x == 64) grid_dep_launch();  // after the epilogue loop, as in the one-CTA kernel
     ptx::tc_fence_before();
     __syncthreads();

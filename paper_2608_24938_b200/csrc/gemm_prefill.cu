@@ -14,6 +14,8 @@
 // then column tile, then row tile, so the CTAs running at the same time share one weight tile
 // through L2 and stream each expert's weights from HBM once. Rows past the end of an expert's
 // group are computed and masked, never padded in memory.
+#include <algorithm>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -99,6 +101,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     __shared__ int s_off[kMaxGroups + 1];
     __shared__ int s_ws[kMaxGroups + 1];
     __shared__ int s_exp[kMaxGroups + 1];
+    __shared__ int s_n_pairs;  // odd-tile pass: whole pairs of row tiles over all groups (the other pass's work)
 
     unsigned char* tiles =
         reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -149,11 +152,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     if (!DEC && p.odd_only) {
         // work table of the odd-tile pass: one row tile for every group whose tile count is odd
         if (warp == 0) {
-            int carry = 0;
+            int carry = 0, pairs = 0;
             for (int g0 = 0; g0 < G; g0 += 32) {
                 const int g = g0 + lane;
                 int odd = 0;
-                if (g < G) odd = ((s_off[g + 1] - s_off[g] + kTileM - 1) / kTileM) & 1;
+                if (g < G) {
+                    const int tiles = (s_off[g + 1] - s_off[g] + kTileM - 1) / kTileM;
+                    odd = tiles & 1;
+                    pairs += tiles >> 1;
+                }
                 int incl = odd;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -163,7 +170,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                 if (g < G) s_ws[g] = carry + incl - odd;
                 carry += __shfl_sync(0xffffffffu, incl, 31);
             }
-            if (lane == 0) s_ws[G] = carry;
+            pairs = __reduce_add_sync(0xffffffffu, pairs);
+            if (lane == 0) {
+                s_ws[G] = carry;
+                s_n_pairs = pairs;
+            }
         }
         __syncthreads();
     }
@@ -175,7 +186,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     // Effective grid: with `rounds` items per CTA, ceil(total / rounds) CTAs finish together; the rest
     // stay idle instead of leaving a few CTAs one item behind (448 items on 148 SMs: 112 x 4, not
     // 144 x 3 + 4 x 4). A hundred SMs are enough to saturate HBM when the kernel is memory-bound.
-    const int rounds = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+    // The odd-tile pass beside the CTA-pair pass keeps only the SMs that pass leaves it (the same function of the same
+    // offsets on both sides); the CTAs beyond them leave at once.
+    int grid_ctas = (int)gridDim.x;
+    if (!DEC && p.odd_only && p.side_by_side) {
+        const int n_clusters = (int)gridDim.x >> 1;
+        grid_ctas = 2 * (n_clusters - pair_pass_clusters(s_n_pairs * nt, total, n_clusters));
+    }
+    const int rounds = grid_ctas > 0 ? (total + grid_ctas - 1) / grid_ctas : 0;
     const int eff_grid = rounds > 0 ? (total + rounds - 1) / rounds : 0;
     const int w_begin = (int)blockIdx.x < eff_grid ? (int)blockIdx.x : total;  // idle CTAs see no work
     const int w_stride = eff_grid > 0 ? eff_grid : 1;
@@ -422,11 +440,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
 
 }  // namespace
 
+// whole_tpcs: launch as clusters of two CTAs. The CTAs do not use the cluster; the launch then occupies SMs two at a
+// time, like the CTA-pair kernel it runs beside, and the two grids cannot leave each other half-filled SM pairs.
 template <int MODE, bool DEC>
-static cudaError_t launch_gemm_t(const GroupedGemmParams& p, int grid, cudaStream_t s) {
+static cudaError_t launch_gemm_t(const GroupedGemmParams& p, int grid, cudaStream_t s, bool whole_tpcs = false) {
     cudaError_t err = cudaFuncSetAttribute(grouped_gemm_kernel<MODE, DEC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            kGemmSmem);
     if (err != cudaSuccess) return err;
+    if (whole_tpcs)
+        return launch_pdl_cluster(grouped_gemm_kernel<MODE, DEC>, std::max(2, grid & ~1), kGemmThreads, kGemmSmem, 2, s, p);
     return launch_pdl(grouped_gemm_kernel<MODE, DEC>, grid, kGemmThreads, kGemmSmem, s, p);
 }
 
@@ -435,6 +457,12 @@ cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStrea
 }
 cudaError_t launch_grouped_gemm2(const GroupedGemmParams& p, int grid, cudaStream_t s) {
     return p.grp_expert != nullptr ? launch_gemm_t<1, true>(p, grid, s) : launch_gemm_t<1, false>(p, grid, s);
+}
+cudaError_t launch_grouped_gemm1_odd(const GroupedGemmParams& p, int grid, cudaStream_t s) {
+    return launch_gemm_t<0, false>(p, grid, s, true);
+}
+cudaError_t launch_grouped_gemm2_odd(const GroupedGemmParams& p, int grid, cudaStream_t s) {
+    return launch_gemm_t<1, false>(p, grid, s, true);
 }
 
 }  // namespace exfold
