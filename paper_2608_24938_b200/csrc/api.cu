@@ -414,13 +414,20 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             if (!side.ok) return EXFOLD_ERR_CUDA;
             GroupedGemmParams go1 = g, go2 = g2;
             go1.odd_only = go2.odd_only = 1;
-            g.side_by_side = g2.side_by_side = go1.side_by_side = go2.side_by_side = 1;
+            // The odd-tile pass is launched with about twice the CTAs its expected share of the work needs (its share
+            // is decided on the device, where the tile counts are known): CTAs without work leave at once, but every
+            // one of them has to pass through one of the pass's few SMs first.
+            const double odd_est = std::max<double>(1.0, G / 2.0), pair_est = std::max<double>(1.0, (tiles_est - G / 2.0) / 2.0);
+            const double q_est = sms * odd_est / (odd_est + 2 * 0.73 * pair_est);
+            const int odd_grid = std::min(sms, 2 * (int)std::ceil(q_est) + 8) & ~1;
+            g.side_by_side = g2.side_by_side = go1.side_by_side = go2.side_by_side = odd_grid;
+            g.n_sm_pairs = g2.n_sm_pairs = go1.n_sm_pairs = go2.n_sm_pairs = sms / 2;
             EXFOLD_CUDA(cudaEventRecord(side.fork, s));
             EXFOLD_CUDA(cudaStreamWaitEvent(side.stream, side.fork, 0));
             {
                 ProfScope ps(3, s);
                 { ProfScope pp(12, s); EXFOLD_CUDA(launch_grouped_gemm1_pair(g, sms, s)); }
-                EXFOLD_CUDA(launch_grouped_gemm1_odd(go1, sms, side.stream));
+                EXFOLD_CUDA(launch_grouped_gemm1_odd(go1, odd_grid, side.stream));
                 if (g_prof.on) {
                     EXFOLD_CUDA(cudaEventRecord(side.mid, side.stream));
                     EXFOLD_CUDA(cudaStreamWaitEvent(s, side.mid, 0));
@@ -429,7 +436,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             {
                 ProfScope ps(4, s);
                 { ProfScope pp(13, s); EXFOLD_CUDA(launch_grouped_gemm2_pair(g2, sms, s)); }
-                EXFOLD_CUDA(launch_grouped_gemm2_odd(go2, sms, side.stream));
+                EXFOLD_CUDA(launch_grouped_gemm2_odd(go2, odd_grid, side.stream));
                 EXFOLD_CUDA(cudaEventRecord(side.join, side.stream));
                 EXFOLD_CUDA(cudaStreamWaitEvent(s, side.join, 0));
             }

@@ -273,9 +273,11 @@ struct GroupedGemmParams {
     float* o32;                 // GEMM-2, calibration: unweighted fp32 outputs O32[row][d] (null: the epilogues above)
     int x_rows;                 // GEMM-1: rows of x; a group that reads x directly starts at row (row0 - R) % x_rows
     int odd_only;               // 1: only each group's last row tile, and only if its tile count is odd (the rest ran on CTA pairs)
-    int side_by_side;           // 1: the CTA-pair pass and the odd-tile pass run at the same time (two streams), both
-                                //    launched over all SMs; each keeps its share of SM pairs (pair_pass_clusters) and
-                                //    the CTAs beyond it leave at once
+    int side_by_side;           // > 0: the CTA-pair pass and the odd-tile pass run at the same time (two streams); the
+                                //    value is the number of CTAs the odd-tile pass was launched with (even). The pair
+                                //    pass is launched over all SMs; each pass keeps its share of SM pairs
+                                //    (pair_pass_clusters) and the CTAs beyond it leave at once
+    int n_sm_pairs;             // side by side: SM pairs the pair pass is launched over (its grid / 2)
     DeviceStatus* status;
 };
 // SM pairs, of n_clusters, that the CTA-pair pass keeps when the odd-tile pass runs beside it on the other
@@ -283,12 +285,14 @@ struct GroupedGemmParams {
 // Side by side, a pair item takes a cluster ~0.73 of the time an odd item takes one SM (measured on the Mixtral shape:
 // 25.9 against 35.7 us per 64-k-block item; the one-CTA kernel is the hungrier of the two for L2 bandwidth and slows
 // down more beside the other); the choice minimises the longer of the two passes, counted in rounds of items.
-__host__ __device__ inline int pair_pass_clusters(int pair_items, int odd_items, int n_clusters) {
+// The odd-tile pass cannot get more than the odd_ctas CTAs it was launched with.
+__host__ __device__ inline int pair_pass_clusters(int pair_items, int odd_items, int n_clusters, int odd_ctas) {
     if (odd_items <= 0) return n_clusters;
-    if (pair_items <= 0) return 0;
-    int best = 1;
+    const int p_min = n_clusters - odd_ctas / 2 > 0 ? n_clusters - odd_ctas / 2 : 0;
+    if (pair_items <= 0) return p_min;
+    int best = p_min > 1 ? p_min : 1;
     float best_t = 3.0e38f;
-    for (int P = 1; P < n_clusters; ++P) {
+    for (int P = best; P < n_clusters; ++P) {
         const int Q = 2 * (n_clusters - P);
         const float tp = 0.73f * (float)((pair_items + P - 1) / P), to = (float)((odd_items + Q - 1) / Q);
         const float t = tp > to ? tp : to;

@@ -100,7 +100,10 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
         abort_s = 0;
         ptx::fence_mbar_init();
     }
-    if (warp == 1) {
+    // Beside the odd-tile pass this kernel is launched over all SMs and the clusters beyond its share must leave
+    // quickly (the other pass waits for their SMs): tensor memory is then allocated only once a cluster knows that
+    // it has work.
+    if (warp == 1 && !p.side_by_side) {
         ptx::tmem_alloc_pair(&tmem_base_s, kPTmemCols);
         ptx::tmem_relinquish_pair();
     }
@@ -138,17 +141,27 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
         }
     }
     __syncthreads();
-    ptx::cluster_sync_all();  // both CTAs' barriers are initialised and their tensor memory allocated
-    ptx::tc_fence_after();
-    const uint32_t tmem_base = tmem_base_s;
     const int nt = p.n_ntiles;
     const int total = s_wp[G] * nt;
     // beside the odd-tile pass this pass keeps only its share of the SM pairs; the other clusters leave at once
-    const int n_pairs = p.side_by_side ? pair_pass_clusters(total, s_n_odd * nt, n_launched) : n_launched;
+    // (both CTAs of a cluster take the same decision: nothing allocated, no cluster barrier entered)
+    const int n_pairs = p.side_by_side ? pair_pass_clusters(total, s_n_odd * nt, n_launched, p.side_by_side) : n_launched;
     const int rounds = n_pairs > 0 ? (total + n_pairs - 1) / n_pairs : 0;
     const int eff = rounds > 0 ? (total + rounds - 1) / rounds : 0;  // pairs that take work and finish together
     const int w_begin = pair_id < eff ? pair_id : total;
     const int w_stride = eff > 0 ? eff : 1;
+    if (p.side_by_side) {
+        if (pair_id >= eff) return;
+        if (warp == 1) {
+            ptx::tmem_alloc_pair(&tmem_base_s, kPTmemCols);
+            ptx::tmem_relinquish_pair();
+        }
+        ptx::tc_fence_before();
+        __syncthreads();
+    }
+    ptx::cluster_sync_all();  // both CTAs' barriers are initialised and their tensor memory allocated
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
     const int nkb = (MODE == 0 ? p.d : p.I) / kPBK;
     volatile int* abort_flag = &abort_s;
 

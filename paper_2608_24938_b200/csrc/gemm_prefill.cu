@@ -131,7 +131,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         abort_s = 0;
         ptx::fence_mbar_init();
     }
-    if (warp == 1) {
+    // The odd-tile pass beside the CTA-pair pass is launched over all SMs and most of its CTAs have nothing to do:
+    // they must leave quickly (they queue for the few SMs of this pass), so tensor memory is allocated only once a
+    // CTA knows that it has work.
+    const bool late_alloc = !DEC && p.odd_only && p.side_by_side;
+    if (warp == 1 && !late_alloc) {
         ptx::tmem_alloc(&tmem_base_s, kTmemCols);
         ptx::tmem_relinquish();
     }
@@ -179,7 +183,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         __syncthreads();
     }
     ptx::tc_fence_after();
-    const uint32_t tmem_base = tmem_base_s;
     const int nt = p.n_ntiles;
     const int ks = (DEC && MODE == 1) ? p.ksplit : 1;  // K parts per tile (needs the fp32-reduction epilogue)
     const int total = s_ws[G] * nt * ks;
@@ -190,13 +193,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     // offsets on both sides); the CTAs beyond them leave at once.
     int grid_ctas = (int)gridDim.x;
     if (!DEC && p.odd_only && p.side_by_side) {
-        const int n_clusters = (int)gridDim.x >> 1;
-        grid_ctas = 2 * (n_clusters - pair_pass_clusters(s_n_pairs * nt, total, n_clusters));
+        // p.n_sm_pairs: SM pairs the pair pass was launched over (this grid may be smaller)
+        grid_ctas = 2 * (p.n_sm_pairs - pair_pass_clusters(s_n_pairs * nt, total, p.n_sm_pairs, (int)gridDim.x));
     }
     const int rounds = grid_ctas > 0 ? (total + grid_ctas - 1) / grid_ctas : 0;
     const int eff_grid = rounds > 0 ? (total + rounds - 1) / rounds : 0;
     const int w_begin = (int)blockIdx.x < eff_grid ? (int)blockIdx.x : total;  // idle CTAs see no work
     const int w_stride = eff_grid > 0 ? eff_grid : 1;
+    if (late_alloc) {
+        if ((int)blockIdx.x >= eff_grid) return;  // the whole CTA: nothing allocated, nothing in flight
+        if (warp == 1) {
+            ptx::tmem_alloc(&tmem_base_s, kTmemCols);
+            ptx::tmem_relinquish();
+        }
+        ptx::tc_fence_before();
+        __syncthreads();
+        ptx::tc_fence_after();
+    }
+    const uint32_t tmem_base = tmem_base_s;
     const int nkb = (MODE == 0 ? p.d : p.I) / kBK;
     const int kb_per = (nkb + ks - 1) / ks;
     // Stage geometry. Prefill: 16 KB A + 32 KB B, 4 stages (compile-time). Decode: the A box has only
