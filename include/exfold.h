@@ -160,11 +160,13 @@ int exfold_calibrate_layers(const exfold_layer *layer, const exfold_calib_job *j
  * routes only). x [T][d], logits [T][N] -> y [T][d]. k_pre = K' in [1, K]; k_pre = K is the
  * unfolded layer. Each token executes exactly K' routed experts (+ the shared expert).
  * Ranking uses key = logit + lnh[e] (one fp32 add; same order as a_e h_e).
- * bf16 layers: the two grouped GEMMs of a large call (>= 48 row tiles of 128 sorted rows, few of them odd last
- * tiles of an expert) run the experts' row tiles two at a time on pairs of CTAs and the odd last tiles on the
- * one-CTA-per-tile kernel; smaller calls use the latter alone. The results are bit-identical either way. The
- * environment variable EXFOLD_PAIR_GEMM (read at every call; 0 = never pairs, 2 = pairs whenever a pair of row
- * tiles exists) overrides the choice; it exists for tests and measurements.
+ * bf16 layers: the two grouped GEMMs of a call of >= 24 row tiles (128 sorted rows each) run the experts' row tiles
+ * two at a time on pairs of CTAs and, beside them, the experts' odd last tiles on the one-CTA-per-tile kernel;
+ * smaller calls use the latter alone. The results are bit-identical either way. The odd-tile kernels run on a
+ * second stream that the library creates once per host thread; they are ordered after the caller's earlier work and
+ * before its later work by events on the caller's stream (also under stream capture). The environment variable
+ * EXFOLD_PAIR_GEMM (read at every call; 0 = never pairs, 2 = pairs whenever a pair of row tiles exists) overrides
+ * the choice; it exists for tests and measurements.
  */
 int exfold_moe_prefill(const exfold_layer *layer, const void *x, const float *logits, int64_t T,
                        const void *w_gate, const void *w_up, const void *w_down,
