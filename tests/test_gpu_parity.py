@@ -248,6 +248,34 @@ def test_prefill_on_cta_pairs_matches_oracle_and_the_one_cta_kernel(shape, monke
         assert np.array_equal(got_pair["y"], got_one["y"])   # bf16 values widened to float32: exact comparison
 
 
+def test_prefill_with_side_by_side_passes_replays_from_a_cuda_graph():
+    """A prefill call whose GEMMs fork onto the library's second stream is captured into a CUDA graph (the fork and
+    the join are events on the capturing stream) and replays to the same bits as the direct call."""
+    cfg = small_bf16(n_experts=4, hidden=256, inter=256, top_k=2, prefill_tokens=2048, logits="normal")  # 32 row tiles
+    case = Case(cfg)
+    ex, T = case.ex, cfg.prefill_tokens
+    ws = case.workspace(T, 2)
+    y_direct = torch.empty((T, cfg.hidden), dtype=case.d_wg.dtype, device=case.dev)
+    y_graph = torch.full_like(y_direct, float("nan"))
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for y in (y_direct, y_direct):   # the second call runs with every lazily created object in place
+            ex.exfold_moe_prefill(case.layer, case.d_x, case.d_lg, case.d_wg, case.d_wu, case.d_wd, case.tables, 2, y, ws,
+                                  stream=stream)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            ex.exfold_moe_prefill(case.layer, case.d_x, case.d_lg, case.d_wg, case.d_wu, case.d_wd, case.tables, 2, y_graph,
+                                  ws, stream=stream)
+        for _ in range(3):
+            graph.replay()
+        stream.synchronize()
+    assert ex.exfold_device_status(ws) == 0
+    assert torch.equal(y_direct.view(torch.int16), y_graph.view(torch.int16))
+    ref = case.oracle_prefill(2)
+    check_output(y_graph.float().cpu().numpy(), ref["y"], "bf16")
+
+
 @pytest.mark.parametrize("T", [1, 63, 129])
 def test_bf16_odd_token_counts(T):
     cfg = small_bf16(prefill_tokens=T, decode_batch=min(T, 256))
