@@ -420,8 +420,8 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             const double odd_est = std::max<double>(1.0, G / 2.0), pair_est = std::max<double>(1.0, (tiles_est - G / 2.0) / 2.0);
             const double q_est = sms * odd_est / (odd_est + 2 * 0.73 * pair_est);
             const int odd_grid = std::min(sms, 2 * (int)std::ceil(q_est) + 8) & ~1;
-            g.side_by_side = g2.side_by_side = go1.side_by_side = go2.side_by_side = odd_grid;
-            g.n_sm_pairs = g2.n_sm_pairs = go1.n_sm_pairs = go2.n_sm_pairs = sms / 2;
+            const SideBySide sbs{nt1, d / kGemmBK, nt2, I / kGemmBK, sms / 2, odd_grid};
+            g.sbs = g2.sbs = go1.sbs = go2.sbs = sbs;
             EXFOLD_CUDA(cudaEventRecord(side.fork, s));
             EXFOLD_CUDA(cudaStreamWaitEvent(side.stream, side.fork, 0));
             {

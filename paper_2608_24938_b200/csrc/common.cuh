@@ -247,6 +247,38 @@ cudaError_t launch_iota_ids(int32_t* ids, int64_t m, int N, cudaStream_t s);
 cudaError_t launch_calib_common_rows(int32_t* offsets, int32_t* work_start, int64_t m, int N, cudaStream_t s);
 
 // ---------------------------------------------------------------- tcgen05 grouped GEMMs (bf16)
+// SM pairs, of n_clusters, that the CTA-pair passes keep when the odd-tile passes run beside them on the other
+// 2 * (n_clusters - P) SMs. Every kernel of a call (both passes of both GEMMs) evaluates this on the device from the
+// same group offsets, so they agree, and the split is the same for GEMM-1 and GEMM-2: `pairs` whole pairs of row tiles
+// and `odd` odd tiles, each times the column tiles (nt) and k-blocks per item (nkb) of the two GEMMs. Side by side,
+// a pair item takes a cluster ~0.73 of the time an odd item takes one SM (measured on the Mixtral shape: 25.9 against
+// 35.7 us per 64-k-block item; the one-CTA kernel is the hungrier of the two for L2 bandwidth and slows down more
+// beside the other). The choice minimises the longer of the two chains (GEMM-1 pass, then GEMM-2 pass), each pass
+// counted in rounds of items. The odd-tile pass cannot get more than the odd_ctas CTAs it was launched with.
+struct SideBySide {
+    int nt1, nkb1, nt2, nkb2;  // column tiles and k-blocks per work item of GEMM-1 and GEMM-2
+    int n_sm_pairs;            // SM pairs the pair passes are launched over
+    int odd_ctas;              // CTAs the odd-tile passes are launched with (even); 0: the passes do not run side by side
+};
+__host__ __device__ inline int pair_pass_clusters(int pairs, int odd, const SideBySide& sb) {
+    const int n = sb.n_sm_pairs;
+    if (odd <= 0) return n;
+    const int p_min = n - sb.odd_ctas / 2 > 0 ? n - sb.odd_ctas / 2 : 0;
+    if (pairs <= 0) return p_min;
+    int best = p_min > 1 ? p_min : 1;
+    float best_t = 3.0e38f;
+    for (int P = best; P < n; ++P) {
+        const int Q = 2 * (n - P);
+        const float tp = 0.73f * (float)(((pairs * sb.nt1 + P - 1) / P) * sb.nkb1 + ((pairs * sb.nt2 + P - 1) / P) * sb.nkb2);
+        const float to = (float)(((odd * sb.nt1 + Q - 1) / Q) * sb.nkb1 + ((odd * sb.nt2 + Q - 1) / Q) * sb.nkb2);
+        const float t = tp > to ? tp : to;
+        if (t < best_t) {
+            best_t = t;
+            best = P;
+        }
+    }
+    return best;
+}
 struct GroupedGemmParams {
     CUtensorMap tm_a;    // GEMM-1: gathered rows Xs [R][d]; GEMM-2: H [Rtot][I]
     CUtensorMap tm_a2;   // GEMM-1: x [T][d] for the shared expert's rows
@@ -273,36 +305,11 @@ struct GroupedGemmParams {
     float* o32;                 // GEMM-2, calibration: unweighted fp32 outputs O32[row][d] (null: the epilogues above)
     int x_rows;                 // GEMM-1: rows of x; a group that reads x directly starts at row (row0 - R) % x_rows
     int odd_only;               // 1: only each group's last row tile, and only if its tile count is odd (the rest ran on CTA pairs)
-    int side_by_side;           // > 0: the CTA-pair pass and the odd-tile pass run at the same time (two streams); the
-                                //    value is the number of CTAs the odd-tile pass was launched with (even). The pair
-                                //    pass is launched over all SMs; each pass keeps its share of SM pairs
-                                //    (pair_pass_clusters) and the CTAs beyond it leave at once
-    int n_sm_pairs;             // side by side: SM pairs the pair pass is launched over (its grid / 2)
+    SideBySide sbs;             // odd_ctas > 0: the CTA-pair pass and the odd-tile pass run at the same time (two
+                                //    streams); each keeps its share of the SM pairs (pair_pass_clusters) and the CTAs
+                                //    beyond it leave at once
     DeviceStatus* status;
 };
-// SM pairs, of n_clusters, that the CTA-pair pass keeps when the odd-tile pass runs beside it on the other
-// 2 * (n_clusters - P) SMs. Both kernels evaluate this on the device from the same group offsets, so they agree.
-// Side by side, a pair item takes a cluster ~0.73 of the time an odd item takes one SM (measured on the Mixtral shape:
-// 25.9 against 35.7 us per 64-k-block item; the one-CTA kernel is the hungrier of the two for L2 bandwidth and slows
-// down more beside the other); the choice minimises the longer of the two passes, counted in rounds of items.
-// The odd-tile pass cannot get more than the odd_ctas CTAs it was launched with.
-__host__ __device__ inline int pair_pass_clusters(int pair_items, int odd_items, int n_clusters, int odd_ctas) {
-    if (odd_items <= 0) return n_clusters;
-    const int p_min = n_clusters - odd_ctas / 2 > 0 ? n_clusters - odd_ctas / 2 : 0;
-    if (pair_items <= 0) return p_min;
-    int best = p_min > 1 ? p_min : 1;
-    float best_t = 3.0e38f;
-    for (int P = best; P < n_clusters; ++P) {
-        const int Q = 2 * (n_clusters - P);
-        const float tp = 0.73f * (float)((pair_items + P - 1) / P), to = (float)((odd_items + Q - 1) / Q);
-        const float t = tp > to ? tp : to;
-        if (t < best_t) {
-            best_t = t;
-            best = P;
-        }
-    }
-    return best;
-}
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s);
 cudaError_t launch_grouped_gemm2(const GroupedGemmParams& p, int grid, cudaStream_t s);
 // Prefill on CTA pairs: every group's row tiles two at a time (a last odd tile is left to the kernels above with

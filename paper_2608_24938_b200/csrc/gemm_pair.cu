@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
     // Beside the odd-tile pass this kernel is launched over all SMs and the clusters beyond its share must leave
     // quickly (the other pass waits for their SMs): tensor memory is then allocated only once a cluster knows that
     // it has work.
-    if (warp == 1 && !p.side_by_side) {
+    if (warp == 1 && p.sbs.odd_ctas == 0) {
         ptx::tmem_alloc_pair(&tmem_base_s, kPTmemCols);
         ptx::tmem_relinquish_pair();
     }
@@ -145,12 +145,13 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
     const int total = s_wp[G] * nt;
     // beside the odd-tile pass this pass keeps only its share of the SM pairs; the other clusters leave at once
     // (both CTAs of a cluster take the same decision: nothing allocated, no cluster barrier entered)
-    const int n_pairs = p.side_by_side ? pair_pass_clusters(total, s_n_odd * nt, n_launched, p.side_by_side) : n_launched;
+    const bool side = p.sbs.odd_ctas > 0;
+    const int n_pairs = side ? pair_pass_clusters(s_wp[G], s_n_odd, p.sbs) : n_launched;
     const int rounds = n_pairs > 0 ? (total + n_pairs - 1) / n_pairs : 0;
     const int eff = rounds > 0 ? (total + rounds - 1) / rounds : 0;  // pairs that take work and finish together
     const int w_begin = pair_id < eff ? pair_id : total;
     const int w_stride = eff > 0 ? eff : 1;
-    if (p.side_by_side) {
+    if (side) {
         if (pair_id >= eff) return;
         if (warp == 1) {
             ptx::tmem_alloc_pair(&tmem_base_s, kPTmemCols);

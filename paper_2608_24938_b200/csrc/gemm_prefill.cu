@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     // The odd-tile pass beside the CTA-pair pass is launched over all SMs and most of its CTAs have nothing to do:
     // they must leave quickly (they queue for the few SMs of this pass), so tensor memory is allocated only once a
     // CTA knows that it has work.
-    const bool late_alloc = !DEC && p.odd_only && p.side_by_side;
+    const bool late_alloc = !DEC && p.odd_only && p.sbs.odd_ctas > 0;
     if (warp == 1 && !late_alloc) {
         ptx::tmem_alloc(&tmem_base_s, kTmemCols);
         ptx::tmem_relinquish();
@@ -192,10 +192,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     // The odd-tile pass beside the CTA-pair pass keeps only the SMs that pass leaves it (the same function of the same
     // offsets on both sides); the CTAs beyond them leave at once.
     int grid_ctas = (int)gridDim.x;
-    if (!DEC && p.odd_only && p.side_by_side) {
-        // p.n_sm_pairs: SM pairs the pair pass was launched over (this grid may be smaller)
-        grid_ctas = 2 * (p.n_sm_pairs - pair_pass_clusters(s_n_pairs * nt, total, p.n_sm_pairs, (int)gridDim.x));
-    }
+    if (late_alloc) grid_ctas = 2 * (p.sbs.n_sm_pairs - pair_pass_clusters(s_n_pairs, s_ws[G], p.sbs));
     const int rounds = grid_ctas > 0 ? (total + grid_ctas - 1) / grid_ctas : 0;
     const int eff_grid = rounds > 0 ? (total + rounds - 1) / rounds : 0;
     const int w_begin = (int)blockIdx.x < eff_grid ? (int)blockIdx.x : total;  // idle CTAs see no work
