@@ -290,39 +290,81 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                 const uint32_t d_tmem = tmem_base + as * 256;
                 const int kpart = ks == 1 ? 0 : w % ks;
                 const int kb0 = kpart * kb_per, kb1 = min(nkb, kb0 + kb_per);
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!ready) {
-                        EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3));
-                        if (!got) {
-                            ok = false;
-                            break;
-                        }
-                    }
-                    if (iter == 0 && kb == kb0) EXFOLD_TRACE_SET(kTr, 9, ptx::globaltimer_ns());
 #ifdef EXFOLD_TRACE
-                    // one CTA of the chosen prefill GEMM logs when each k-block's operands were ready (cycles; the
-                    // ns timer once per 16 k-blocks, for the clock rate)
+                // one CTA of the chosen prefill GEMM logs when each k-block's (EXFOLD_TRACE_TILE: work item's) operands
+                // were ready: cycles, and the ns timer with every 16th entry (for the clock rate)
 #ifdef EXFOLD_TRACE_PAIR
-                    if (false) {
+#define EXFOLD_KB_TRACE_COND false
 #elif defined(EXFOLD_TRACE_TILE)
-                    if (MODE == EXFOLD_TRACE_KB_MODE && !DEC && blockIdx.x == 5 && kbt < kTraceKb && kb == kb0) {
+#define EXFOLD_KB_TRACE_COND (kb == kb0)
 #else
-                    if (MODE == EXFOLD_TRACE_KB_MODE && !DEC && blockIdx.x == 5 && kbt < kTraceKb) {
+#define EXFOLD_KB_TRACE_COND true
 #endif
-                        unsigned long long* flat = &g_trace[3][0][0];
-                        flat[kbt] = (unsigned long long)clock64();
-                        if ((kbt & 15) == 0) flat[kTraceKb + kbt] = ptx::globaltimer_ns();
-                        ++kbt;
+#define EXFOLD_KB_TRACE()                                                                                     \
+    do {                                                                                                      \
+        if (MODE == EXFOLD_TRACE_KB_MODE && !DEC && blockIdx.x == 5 && kbt < kTraceKb && EXFOLD_KB_TRACE_COND) { \
+            unsigned long long* flat = &g_trace[3][0][0];                                                     \
+            flat[kbt] = (unsigned long long)clock64();                                                        \
+            if ((kbt & 15) == 0) flat[kTraceKb + kbt] = ptx::globaltimer_ns();                                \
+            ++kbt;                                                                                            \
+        }                                                                                                     \
+    } while (0)
+#else
+#define EXFOLD_KB_TRACE() ((void)0)
+#endif
+                if constexpr (!DEC && kStages == 4) {
+                    // Prefill: the k-loop is written out once per ring stage (switch into the stage the ring stands
+                    // at), so a k-block costs this thread the MMA sequence, one compare and one branch.
+                    int kb = kb0;
+#define EXFOLD_KBLOCK(S)                                                                                            \
+    {                                                                                                                \
+        constexpr int NS = (S) + 1 == kStages ? 0 : (S) + 1;                                                         \
+        const uint32_t nphase = NS == 0 ? phase ^ 1 : phase;                                                         \
+        if (!ready && !ptx::mbar_wait(&full_bar[S], phase, abort_flag, p.status, 3)) {                               \
+            ok = false;                                                                                              \
+            break;                                                                                                   \
+        }                                                                                                            \
+        EXFOLD_KB_TRACE();                                                                                           \
+        constexpr uint32_t step = (uint32_t)kStageBytes >> 4, off_b = (uint32_t)kATileBytes >> 4;                    \
+        ready = ptx::umma_kblock_bf16(d_tmem, lo0 + (S) * step, lo0 + (S) * step + off_b, desc_hi32, idesc,         \
+                                      kb > kb0 ? 1u : 0u, &empty_bar[S], &full_bar[NS], nphase);                     \
+        if (NS == 0) phase ^= 1;                                                                                     \
+        if (++kb == kb1) {                                                                                           \
+            stage = NS;                                                                                              \
+            break;                                                                                                   \
+        }                                                                                                            \
+    }
+                    while (ok && kb < kb1) {
+                        switch (stage) {
+                            case 0: EXFOLD_KBLOCK(0)
+                            case 1: EXFOLD_KBLOCK(1)
+                            case 2: EXFOLD_KBLOCK(2)
+                            default: EXFOLD_KBLOCK(3)
+                        }
+                        if (kb < kb1) stage = 0;  // fell through the last stage: the ring wraps
                     }
-#endif
-                    const int ns = stage + 1 == stages ? 0 : stage + 1;
-                    const int nphase = ns == 0 ? phase ^ 1 : phase;
-                    ready = ptx::umma_kblock_bf16(d_tmem, a_lo, a_lo + lo_b, desc_hi32, idesc, kb > kb0 ? 1u : 0u,
-                                                  &empty_bar[stage], &full_bar[ns], nphase);
-                    a_lo = ns == 0 ? lo0 : a_lo + lo_step;
-                    stage = ns;
-                    phase = nphase;
+#undef EXFOLD_KBLOCK
+                } else {
+                    for (int kb = kb0; kb < kb1; ++kb) {
+                        if (!ready) {
+                            EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3));
+                            if (!got) {
+                                ok = false;
+                                break;
+                            }
+                        }
+                        if (iter == 0 && kb == kb0) EXFOLD_TRACE_SET(kTr, 9, ptx::globaltimer_ns());
+                        EXFOLD_KB_TRACE();
+                        const int ns = stage + 1 == stages ? 0 : stage + 1;
+                        const int nphase = ns == 0 ? phase ^ 1 : phase;
+                        ready = ptx::umma_kblock_bf16(d_tmem, a_lo, a_lo + lo_b, desc_hi32, idesc, kb > kb0 ? 1u : 0u,
+                                                      &empty_bar[stage], &full_bar[ns], nphase);
+                        a_lo = ns == 0 ? lo0 : a_lo + lo_step;
+                        stage = ns;
+                        phase = nphase;
+                    }
                 }
+#undef EXFOLD_KB_TRACE
                 if (ok) ptx::umma_commit(&tfull_bar[as]);
             }
             EXFOLD_TRACE_SET(kTr, 5, tr_wait);
