@@ -184,22 +184,41 @@ int pair_gemm_mode() {
 }
 
 // Second stream (and fork / join events) on which the odd-tile passes of a prefill call run beside the CTA-pair
-// passes. Created once per host thread, on first use, and kept for the life of the process.
+// passes. Created once per host thread and device, on first use, and kept for the life of the process.
 struct SideStream {
     cudaStream_t stream = nullptr;
     cudaEvent_t fork = nullptr, join = nullptr, mid = nullptr;
     bool ok = false;
 };
-SideStream& side_stream() {
-    static thread_local SideStream h;
+constexpr int kMaxDevices = 64;
+SideStream* side_stream() {
+    static thread_local SideStream per_device[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    SideStream& h = per_device[dev];
     if (!h.ok) {
         h.ok = cudaStreamCreateWithFlags(&h.stream, cudaStreamNonBlocking) == cudaSuccess &&
                cudaEventCreateWithFlags(&h.fork, cudaEventDisableTiming) == cudaSuccess &&
                cudaEventCreateWithFlags(&h.join, cudaEventDisableTiming) == cudaSuccess &&
                cudaEventCreateWithFlags(&h.mid, cudaEventDisableTiming) == cudaSuccess;
     }
-    return h;
+    return h.ok ? &h : nullptr;
 }
+// Once the side stream has been forked off the caller's stream it is joined again on every way out of the call
+// (also the error returns): later work on the caller's stream, or the end of a stream capture, must not overtake it.
+struct SideJoin {
+    SideStream* side;
+    cudaStream_t s;
+    bool armed = true;
+    cudaError_t join() {
+        armed = false;
+        cudaError_t e = cudaEventRecord(side->join, side->stream);
+        return e != cudaSuccess ? e : cudaStreamWaitEvent(s, side->join, 0);
+    }
+    ~SideJoin() {
+        if (armed) join();
+    }
+};
 
 int sm_count() {
     static int n = 0;
@@ -410,8 +429,9 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             // of GEMM-2 follows the same pass of GEMM-1 on its own stream: caller's stream: GEMM-1 pairs -> GEMM-2
             // pairs; side stream: GEMM-1 odd tiles -> GEMM-2 odd tiles; joined before the combine kernel (or the
             // end of the call). With per-kernel timing on, the streams also join between the two GEMMs.
-            SideStream& side = side_stream();
-            if (!side.ok) return EXFOLD_ERR_CUDA;
+            SideStream* sidep = side_stream();
+            if (!sidep) return EXFOLD_ERR_CUDA;
+            SideStream& side = *sidep;
             GroupedGemmParams go1 = g, go2 = g2;
             go1.odd_only = go2.odd_only = 1;
             // The odd-tile pass is launched with about twice the CTAs its expected share of the work needs (its share
@@ -424,6 +444,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             g.sbs = g2.sbs = go1.sbs = go2.sbs = sbs;
             EXFOLD_CUDA(cudaEventRecord(side.fork, s));
             EXFOLD_CUDA(cudaStreamWaitEvent(side.stream, side.fork, 0));
+            SideJoin joiner{sidep, s};
             {
                 ProfScope ps(3, s);
                 { ProfScope pp(12, s); EXFOLD_CUDA(launch_grouped_gemm1_pair(g, sms, s)); }
@@ -437,8 +458,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
                 ProfScope ps(4, s);
                 { ProfScope pp(13, s); EXFOLD_CUDA(launch_grouped_gemm2_pair(g2, sms, s)); }
                 EXFOLD_CUDA(launch_grouped_gemm2_odd(go2, odd_grid, side.stream));
-                EXFOLD_CUDA(cudaEventRecord(side.join, side.stream));
-                EXFOLD_CUDA(cudaStreamWaitEvent(s, side.join, 0));
+                EXFOLD_CUDA(joiner.join());
             }
         }
         if (!direct) {
