@@ -18,9 +18,17 @@
  *     any, is expert index N. x, W_*, y have the layer dtype; router logits and all
  *     tables are fp32; indices are int32.
  *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the
- *     caller. The library allocates no device memory and keeps no state between calls:
- *     all scratch lives in the caller's workspace `ws` (exfold_workspace_bytes; 256-byte
- *     aligned). Calls that share a workspace must be ordered on one stream.
+ *     caller. The library allocates no device memory: all scratch lives in the caller's
+ *     workspace `ws` (exfold_workspace_bytes; 256-byte aligned). Calls that share a
+ *     workspace must be ordered on one stream.
+ *   - What the library keeps between calls, and nothing else: (a) per host thread and device,
+ *     created on first use and freed by exfold_thread_release: one extra CUDA stream with three
+ *     events (large prefill calls run two kernel chains side by side on it) and two copy streams
+ *     with ten events (chunked host-buffer prefill). Calls issued by one host thread on
+ *     different caller streams share them, so the parts that use them run one after the other;
+ *     results do not depend on it. (b) per process: the launch counter, the optional
+ *     per-kernel timing events (exfold_profile_*, off by default, not thread-safe) and the
+ *     built-in scratch array of exfold_moe_decode_noalloc. No environment variable is read.
  *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
  *     default stream) and return without synchronising, except exfold_device_status.
  *   - Return value: EXFOLD_OK (0), a negative error (nothing was launched), or a positive
@@ -164,9 +172,8 @@ int exfold_calibrate_layers(const exfold_layer *layer, const exfold_calib_job *j
  * two at a time on pairs of CTAs and, beside them, the experts' odd last tiles on the one-CTA-per-tile kernel;
  * smaller calls use the latter alone. The results are bit-identical either way. The odd-tile kernels run on a
  * second stream that the library creates once per host thread; they are ordered after the caller's earlier work and
- * before its later work by events on the caller's stream (also under stream capture). The environment variable
- * EXFOLD_PAIR_GEMM (read at every call; 0 = never pairs, 2 = pairs whenever a pair of row tiles exists) overrides
- * the choice; it exists for tests and measurements.
+ * before its later work by events on the caller's stream (also under stream capture). exfold_fold_opts.gemm_path
+ * overrides the choice of kernels (tests and measurements).
  */
 int exfold_moe_prefill(const exfold_layer *layer, const void *x, const float *logits, int64_t T,
                        const void *w_gate, const void *w_up, const void *w_down,
@@ -185,11 +192,14 @@ int exfold_moe_prefill(const exfold_layer *layer, const void *x, const float *lo
  *   confidence_split  != 0: with c = clip(1 - L[s][t], 0, 1) for the minimum-loss target t, the part
  *                     w_s c S[s][t] is folded onto t and w_s (1 - c) is spread over the retained
  *                     routes in proportion to their original router weights.
+ *   gemm_path         0: the library chooses the tensor-core kernels (above); 1: one-CTA kernel only;
+ *                     2: CTA pairs wherever a group has a pair of row tiles. Same results bit for bit.
  */
 typedef struct {
     float loss_threshold;
     int32_t rescale;
     int32_t confidence_split;
+    int32_t gemm_path;
 } exfold_fold_opts;
 
 int exfold_moe_prefill_ex(const exfold_layer *layer, const void *x, const float *logits, int64_t T,
@@ -255,7 +265,7 @@ int exfold_router_logits(const exfold_layer *layer, const void *x, const void *w
  * must be exfold_workspace_bytes(...) + exfold_host_staging_bytes(...) large.
  * A prefill call of 4096 tokens or more that asks for no metadata is run as up to four chunks of whole
  * 128-row tiles: the next chunk is copied in and the previous one copied out on two helper streams
- * created and destroyed inside the call, while the caller's stream computes; the call still completes in
+ * (created once per host thread and device), while the caller's stream computes; the call still completes in
  * the caller's stream order and the result is the same bit for bit (tokens do not interact).
  */
 size_t exfold_host_staging_bytes(const exfold_layer *layer, int64_t max_tokens);
@@ -290,13 +300,21 @@ int exfold_moe_decode_host(const exfold_layer *layer, const void *x_host, const 
  *   - all calls on a device share the one array, which keeps what the previous call left in it;
  *     the call itself clears what must start at zero, but two calls that overlap on the GPU
  *     (different streams, no ordering between them) race on it: keep them on one stream or order
- *     them with events.
+ *     them with events;
+ *   - the status record of these calls sits at the start of that array: read it with
+ *     exfold_device_status_noalloc (same meaning and behaviour as exfold_device_status: it
+ *     synchronises the stream, reports a bounded wait that ran out, and clears the record). Without
+ *     that check a timed-out call goes unnoticed, because the next call clears the record first.
+ * exfold_static_scratch_address writes the array's device address on the current device to
+ * *address (host pointer), for diagnostics and memory checkers; the array is never to be freed.
  */
 #define EXFOLD_STATIC_SCRATCH_BYTES (8u << 20)
 int exfold_moe_decode_noalloc(const exfold_layer *layer, const void *x, const float *logits, int64_t B,
                               const void *w_gate, const void *w_up, const void *w_down,
                               const exfold_tables *tables, int32_t pool_m, void *y,
                               const exfold_decode_meta *meta, void *cuda_stream);
+int exfold_device_status_noalloc(void *cuda_stream);
+int exfold_static_scratch_address(void **address);
 
 /*
  * Synchronises the stream and decodes the status word the kernels keep at the start of the
@@ -304,6 +322,13 @@ int exfold_moe_decode_noalloc(const exfold_layer *layer, const void *x, const fl
  * EXFOLD_ERR_CUDA. Clears the word. The only synchronising call on the serving path.
  */
 int exfold_device_status(void *ws, void *cuda_stream);
+
+/*
+ * Destroys the CUDA streams and events the library created for the calling host thread on the current
+ * device (see the conventions above); they are created again by the next call that needs them. The
+ * caller makes sure none of its calls is still running on them (synchronise first).
+ */
+int exfold_thread_release(void);
 
 /* Human-readable name of a status code (static storage). */
 const char *exfold_status_string(int status);

@@ -30,7 +30,8 @@ EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibr
            "exfold_moe_decode", "exfold_moe_prefill_host", "exfold_moe_decode_host", "exfold_device_status",
            "exfold_status_string", "exfold_launch_count", "exfold_profile_enable", "exfold_profile_read",
            "exfold_moe_decode_noalloc", "exfold_static_pool_build", "exfold_moe_decode_static",
-           "exfold_moe_prefill_ex", "exfold_router_logits", "exfold_calibrate_layers"]
+           "exfold_moe_prefill_ex", "exfold_router_logits", "exfold_calibrate_layers", "exfold_device_status_noalloc",
+           "exfold_static_scratch_address", "exfold_thread_release"]
 PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
                  "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
                  "simt_combine", "gemm1_pair_pass", "gemm2_pair_pass"]
@@ -66,7 +67,8 @@ class exfold_decode_meta(C.Structure):
 
 
 class exfold_fold_opts(C.Structure):
-    _fields_ = [("loss_threshold", C.c_float), ("rescale", C.c_int32), ("confidence_split", C.c_int32)]
+    _fields_ = [("loss_threshold", C.c_float), ("rescale", C.c_int32), ("confidence_split", C.c_int32),
+                ("gemm_path", C.c_int32)]
 
 
 class exfold_static_pool(C.Structure):
@@ -113,6 +115,12 @@ def _load() -> C.CDLL:
                                              C.POINTER(exfold_static_pool), vp, C.POINTER(exfold_decode_meta), vp, sz, vp]
     lib.exfold_device_status.restype = C.c_int
     lib.exfold_device_status.argtypes = [vp, vp]
+    lib.exfold_device_status_noalloc.restype = C.c_int
+    lib.exfold_device_status_noalloc.argtypes = [vp]
+    lib.exfold_static_scratch_address.restype = C.c_int
+    lib.exfold_static_scratch_address.argtypes = [C.POINTER(vp)]
+    lib.exfold_thread_release.restype = C.c_int
+    lib.exfold_thread_release.argtypes = []
     lib.exfold_status_string.restype = C.c_char_p
     lib.exfold_status_string.argtypes = [C.c_int]
     lib.exfold_launch_count.restype = i64
@@ -205,6 +213,22 @@ def exfold_router_logits(layer, x, w_router, logits, ws, stream=None) -> int:
 
 def exfold_device_status(ws: torch.Tensor, stream=None) -> int:
     return int(lib.exfold_device_status(_ptr(ws), _stream(stream)))
+
+
+def exfold_device_status_noalloc(stream=None) -> int:
+    return int(lib.exfold_device_status_noalloc(_stream(stream)))
+
+
+def exfold_static_scratch_address() -> int:
+    out = C.c_void_p()
+    rc = lib.exfold_static_scratch_address(C.byref(out))
+    if rc != 0:
+        raise ExfoldError(rc, "exfold_static_scratch_address")
+    return int(out.value)
+
+
+def exfold_thread_release() -> int:
+    return int(lib.exfold_thread_release())
 
 
 def exfold_calibrate(layer, x_cal, logits_cal, w_gate, w_up, w_down, out: exfold_tables, ws, lam=1e-3,
@@ -324,8 +348,8 @@ def exfold_moe_decode_static(layer, x, logits, w_gate, w_up, w_down, pool: exfol
 
 def exfold_moe_prefill_ex(layer, x, logits, w_gate, w_up, w_down, tables: exfold_tables, k_pre: int, y, ws,
                           loss_threshold: float = float("inf"), rescale: bool = False, confidence_split: bool = False,
-                          meta: Optional[dict] = None, stream=None, check: bool = True) -> int:
-    opts = exfold_fold_opts(loss_threshold, int(rescale), int(confidence_split))
+                          gemm_path: int = 0, meta: Optional[dict] = None, stream=None, check: bool = True) -> int:
+    opts = exfold_fold_opts(loss_threshold, int(rescale), int(confidence_split), int(gemm_path))
     rc = lib.exfold_moe_prefill_ex(C.byref(layer), _ptr(x), _ptr(logits), x.shape[0], _ptr(w_gate), _ptr(w_up),
                                    _ptr(w_down), C.byref(tables), k_pre, C.byref(opts), _ptr(y), _prefill_meta(meta),
                                    _ptr(ws), ws.numel(), _stream(stream))

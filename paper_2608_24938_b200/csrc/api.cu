@@ -10,15 +10,6 @@
 #include "common.cuh"
 #include "ptx.cuh"
 
-#ifdef EXFOLD_TRACE
-namespace exfold {
-__device__ unsigned long long g_trace[4][kMaxCtas][kTraceSlots];
-}
-extern "C" int exfold_debug_read_trace(unsigned long long* out) {  // [4][kMaxCtas][kTraceSlots]
-    cudaDeviceSynchronize();
-    return cudaMemcpyFromSymbol(out, exfold::g_trace, sizeof(exfold::g_trace)) == cudaSuccess ? 0 : -4;
-}
-#endif
 
 namespace exfold {
 
@@ -175,44 +166,66 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, u
     return r == CUDA_SUCCESS;
 }
 
-// EXFOLD_PAIR_GEMM=0 keeps prefill on the one-CTA kernel; =2 takes the CTA-pair kernel whenever a pair can exist
-// (the parity tests run both kernels on small inputs this way); unset or 1: the choice below. Read at every call.
-int pair_gemm_mode() {
-    const char* e = getenv("EXFOLD_PAIR_GEMM");
-    const int mode = e ? atoi(e) : 1;
-    return mode < 0 || mode > 2 ? 1 : mode;
-}
-
-// Second stream (and fork / join events) on which the odd-tile passes of a prefill call run beside the CTA-pair
-// passes. Created once per host thread and device, on first use, and kept for the life of the process.
-struct SideStream {
-    cudaStream_t stream = nullptr;
-    cudaEvent_t fork = nullptr, join = nullptr, mid = nullptr;
-    bool ok = false;
-};
+// Host-side CUDA objects the library keeps per (host thread, device), created on first use and kept until
+// exfold_thread_release() or the end of the process:
+//   side stream + fork / join / mid events: the odd-tile passes of a prefill call run beside the CTA-pair passes;
+//   in / out streams + events: the chunked host-buffer prefill copies the next chunk in and the previous one out
+//   while the caller's stream computes.
+// Nothing else survives a call. Two caller streams used from one host thread share these objects, so the parts of
+// their calls that run on them are ordered one after the other (results are unaffected).
 constexpr int kMaxDevices = 64;
-SideStream* side_stream() {
-    static thread_local SideStream per_device[kMaxDevices];
+struct ThreadDeviceState {
+    cudaStream_t side = nullptr, in = nullptr, out = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr, mid = nullptr;
+    cudaEvent_t start = nullptr, done = nullptr, copied[kMaxHostChunks] = {}, computed[kMaxHostChunks] = {};
+    bool side_ok = false, host_ok = false;
+    int sms = 0;
+    void release() {
+        auto ev = [](cudaEvent_t& e) { if (e) cudaEventDestroy(e); e = nullptr; };
+        auto st = [](cudaStream_t& s) { if (s) cudaStreamDestroy(s); s = nullptr; };
+        ev(fork); ev(join); ev(mid); ev(start); ev(done);
+        for (int c = 0; c < kMaxHostChunks; ++c) { ev(copied[c]); ev(computed[c]); }
+        st(side); st(in); st(out);
+        side_ok = host_ok = false;
+    }
+};
+thread_local ThreadDeviceState t_state[kMaxDevices];
+
+ThreadDeviceState* thread_state() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-    SideStream& h = per_device[dev];
-    if (!h.ok) {
-        h.ok = cudaStreamCreateWithFlags(&h.stream, cudaStreamNonBlocking) == cudaSuccess &&
-               cudaEventCreateWithFlags(&h.fork, cudaEventDisableTiming) == cudaSuccess &&
-               cudaEventCreateWithFlags(&h.join, cudaEventDisableTiming) == cudaSuccess &&
-               cudaEventCreateWithFlags(&h.mid, cudaEventDisableTiming) == cudaSuccess;
+    return &t_state[dev];
+}
+bool new_event(cudaEvent_t* e) { return cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; }
+// second stream (and fork / join events) for the odd-tile passes of a prefill call
+ThreadDeviceState* side_stream() {
+    ThreadDeviceState* h = thread_state();
+    if (h && !h->side_ok)
+        h->side_ok = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) == cudaSuccess && new_event(&h->fork) &&
+                     new_event(&h->join) && new_event(&h->mid);
+    return h && h->side_ok ? h : nullptr;
+}
+// copy-in / copy-out streams and events of the chunked host-buffer prefill
+ThreadDeviceState* host_helpers() {
+    ThreadDeviceState* h = thread_state();
+    if (h && !h->host_ok) {
+        bool ok = cudaStreamCreateWithFlags(&h->in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&h->out, cudaStreamNonBlocking) == cudaSuccess && new_event(&h->start) &&
+                  new_event(&h->done);
+        for (int c = 0; ok && c < kMaxHostChunks; ++c) ok = new_event(&h->copied[c]) && new_event(&h->computed[c]);
+        h->host_ok = ok;
     }
-    return h.ok ? &h : nullptr;
+    return h && h->host_ok ? h : nullptr;
 }
 // Once the side stream has been forked off the caller's stream it is joined again on every way out of the call
 // (also the error returns): later work on the caller's stream, or the end of a stream capture, must not overtake it.
 struct SideJoin {
-    SideStream* side;
+    ThreadDeviceState* side;
     cudaStream_t s;
     bool armed = true;
     cudaError_t join() {
         armed = false;
-        cudaError_t e = cudaEventRecord(side->join, side->stream);
+        cudaError_t e = cudaEventRecord(side->join, side->side);
         return e != cudaSuccess ? e : cudaStreamWaitEvent(s, side->join, 0);
     }
     ~SideJoin() {
@@ -220,13 +233,14 @@ struct SideJoin {
     }
 };
 
-int sm_count() {
-    static int n = 0;
-    if (!n) {
+int sm_count() {  // of the current device
+    ThreadDeviceState* h = thread_state();
+    int n = h ? h->sms : 0;
+    if (n <= 0) {
         int dev = 0;
         cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        if (h) h->sms = n;
     }
     return n;
 }
@@ -258,6 +272,16 @@ int check_common(const exfold_layer* layer, const void* x, const float* logits, 
 }
 
 }  // namespace
+
+// Synchronises the stream, decodes and clears the status record at `rec` (device memory)
+int read_status_record(void* rec, cudaStream_t s) {
+    if (cudaStreamSynchronize(s) != cudaSuccess) return EXFOLD_ERR_CUDA;
+    int code = 0;
+    if (cudaMemcpy(&code, rec, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return EXFOLD_ERR_CUDA;
+    if (cudaMemset(rec, 0, sizeof(DeviceStatus)) != cudaSuccess) return EXFOLD_ERR_CUDA;
+    if (code == 0) return EXFOLD_OK;
+    return code == EXFOLD_ERR_DEVICE_TIMEOUT ? EXFOLD_ERR_DEVICE_TIMEOUT : EXFOLD_ERR_CUDA;
+}
 }  // namespace exfold
 
 using namespace exfold;
@@ -324,13 +348,14 @@ const char* exfold_status_string(int status) {
 
 int exfold_device_status(void* ws, void* cuda_stream) {
     if (!ws) return EXFOLD_ERR_INVALID_ARG;
-    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
-    if (cudaStreamSynchronize(s) != cudaSuccess) return EXFOLD_ERR_CUDA;
-    int code = 0;
-    if (cudaMemcpy(&code, ws, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return EXFOLD_ERR_CUDA;
-    if (cudaMemset(ws, 0, sizeof(DeviceStatus)) != cudaSuccess) return EXFOLD_ERR_CUDA;
-    if (code == 0) return EXFOLD_OK;
-    return code == EXFOLD_ERR_DEVICE_TIMEOUT ? EXFOLD_ERR_DEVICE_TIMEOUT : EXFOLD_ERR_CUDA;
+    return read_status_record(ws, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int exfold_thread_release(void) {
+    ThreadDeviceState* h = thread_state();
+    if (!h) return EXFOLD_ERR_CUDA;
+    h->release();
+    return EXFOLD_OK;
 }
 
 int exfold_moe_prefill(const exfold_layer* layer, const void* x, const float* logits, int64_t T, const void* w_gate,
@@ -364,8 +389,8 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     // Measured against the one-CTA kernel alone: Mixtral shape 4096 / 8192 / 16384 / 32768 tokens -3 / -9 / -14 /
     // -16 %, GLM shape -8 %, Qwen3 shape (half of the experts own a single tile) -1 %.
     const int64_t tiles_est = Rtot / kTileM + G / 2;
-    const int mode = pair_gemm_mode();
-    const bool pairs = bf16 && kGemmBK == 64 && (mode == 2 ? Rtot >= 2 * kTileM : mode == 1 && tiles_est >= 24);
+    const int mode = opts == nullptr || opts->gemm_path < 0 || opts->gemm_path > 2 ? 0 : opts->gemm_path;
+    const bool pairs = bf16 && kGemmBK == 64 && (mode == 2 ? Rtot >= 2 * kTileM : mode == 0 && tiles_est >= 24);
     const int sms = sm_count() & ~1;
     if (bf16) {
         const uint64_t E = (uint64_t)G;
@@ -429,9 +454,9 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             // of GEMM-2 follows the same pass of GEMM-1 on its own stream: caller's stream: GEMM-1 pairs -> GEMM-2
             // pairs; side stream: GEMM-1 odd tiles -> GEMM-2 odd tiles; joined before the combine kernel (or the
             // end of the call). With per-kernel timing on, the streams also join between the two GEMMs.
-            SideStream* sidep = side_stream();
+            ThreadDeviceState* sidep = side_stream();
             if (!sidep) return EXFOLD_ERR_CUDA;
-            SideStream& side = *sidep;
+            ThreadDeviceState& side = *sidep;
             GroupedGemmParams go1 = g, go2 = g2;
             go1.odd_only = go2.odd_only = 1;
             // The odd-tile pass is launched with about twice the CTAs its expected share of the work needs (its share
@@ -443,21 +468,21 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             const SideBySide sbs{nt1, d / kGemmBK, nt2, I / kGemmBK, sms / 2, odd_grid};
             g.sbs = g2.sbs = go1.sbs = go2.sbs = sbs;
             EXFOLD_CUDA(cudaEventRecord(side.fork, s));
-            EXFOLD_CUDA(cudaStreamWaitEvent(side.stream, side.fork, 0));
+            EXFOLD_CUDA(cudaStreamWaitEvent(side.side, side.fork, 0));
             SideJoin joiner{sidep, s};
             {
                 ProfScope ps(3, s);
                 { ProfScope pp(12, s); EXFOLD_CUDA(launch_grouped_gemm1_pair(g, sms, s)); }
-                EXFOLD_CUDA(launch_grouped_gemm1_odd(go1, odd_grid, side.stream));
+                EXFOLD_CUDA(launch_grouped_gemm1_odd(go1, odd_grid, side.side));
                 if (g_prof.on) {
-                    EXFOLD_CUDA(cudaEventRecord(side.mid, side.stream));
+                    EXFOLD_CUDA(cudaEventRecord(side.mid, side.side));
                     EXFOLD_CUDA(cudaStreamWaitEvent(s, side.mid, 0));
                 }
             }
             {
                 ProfScope ps(4, s);
                 { ProfScope pp(13, s); EXFOLD_CUDA(launch_grouped_gemm2_pair(g2, sms, s)); }
-                EXFOLD_CUDA(launch_grouped_gemm2_odd(go2, odd_grid, side.stream));
+                EXFOLD_CUDA(launch_grouped_gemm2_odd(go2, odd_grid, side.side));
                 EXFOLD_CUDA(joiner.join());
             }
         }
@@ -834,6 +859,9 @@ int exfold_moe_prefill_host(const exfold_layer* layer, const void* x_host, const
     // metadata describes the whole call (one permutation over all routes), so a call that asks for it is not split.
     const int64_t chunk_tokens = 2048;
     int chunks = meta != nullptr ? 1 : (int)std::min<int64_t>(kMaxHostChunks, T / chunk_tokens);
+    // a chunk of at least 12 row tiles still runs its whole tile pairs on the CTA-pair kernel
+    const int64_t chunk_rows = chunks > 1 ? (T / chunks) * (k_pre + layer->n_shared) : 0;
+    exfold_fold_opts chunk_opts{INFINITY, 0, 0, chunk_rows >= 12 * kTileM ? 2 : 0};
     if (chunks <= 1) {
         EXFOLD_CUDA(cudaMemcpyAsync(xd, x_host, xb, cudaMemcpyHostToDevice, s));
         EXFOLD_CUDA(cudaMemcpyAsync(ld, logits_host, lb, cudaMemcpyHostToDevice, s));
@@ -843,28 +871,9 @@ int exfold_moe_prefill_host(const exfold_layer* layer, const void* x_host, const
         EXFOLD_CUDA(cudaMemcpyAsync(y_host, yd, xb, cudaMemcpyDeviceToHost, s));
         return EXFOLD_OK;
     }
-    struct Helpers {  // per-call helper streams and events; destruction is deferred by the runtime until they drain
-        cudaStream_t in = nullptr, out = nullptr;
-        cudaEvent_t start = nullptr, copied[kMaxHostChunks] = {}, computed[kMaxHostChunks] = {}, done = nullptr;
-        ~Helpers() {
-            if (start) cudaEventDestroy(start);
-            if (done) cudaEventDestroy(done);
-            for (int c = 0; c < kMaxHostChunks; ++c) {
-                if (copied[c]) cudaEventDestroy(copied[c]);
-                if (computed[c]) cudaEventDestroy(computed[c]);
-            }
-            if (in) cudaStreamDestroy(in);
-            if (out) cudaStreamDestroy(out);
-        }
-    } h;
-    EXFOLD_CUDA(cudaStreamCreateWithFlags(&h.in, cudaStreamNonBlocking));
-    EXFOLD_CUDA(cudaStreamCreateWithFlags(&h.out, cudaStreamNonBlocking));
-    EXFOLD_CUDA(cudaEventCreateWithFlags(&h.start, cudaEventDisableTiming));
-    EXFOLD_CUDA(cudaEventCreateWithFlags(&h.done, cudaEventDisableTiming));
-    for (int c = 0; c < chunks; ++c) {
-        EXFOLD_CUDA(cudaEventCreateWithFlags(&h.copied[c], cudaEventDisableTiming));
-        EXFOLD_CUDA(cudaEventCreateWithFlags(&h.computed[c], cudaEventDisableTiming));
-    }
+    ThreadDeviceState* hp = host_helpers();  // created once per host thread and device
+    if (!hp) return EXFOLD_ERR_CUDA;
+    ThreadDeviceState& h = *hp;
     // the staging buffers may still be in use by earlier work on the caller's stream
     EXFOLD_CUDA(cudaEventRecord(h.start, s));
     EXFOLD_CUDA(cudaStreamWaitEvent(h.in, h.start, 0));
@@ -885,8 +894,9 @@ int exfold_moe_prefill_host(const exfold_layer* layer, const void* x_host, const
         if (n <= 0) break;
         EXFOLD_CUDA(cudaStreamWaitEvent(s, h.copied[c], 0));
         t_keep_status = c > 0;  // an error recorded by an earlier chunk stays visible
-        int rc = exfold_moe_prefill(layer, xd + t0 * row_x, reinterpret_cast<const float*>(ld + t0 * row_l), n, w_gate,
-                                    w_up, w_down, tables, k_pre, yd + t0 * row_x, nullptr, ws, main_bytes, cuda_stream);
+        int rc = exfold_moe_prefill_ex(layer, xd + t0 * row_x, reinterpret_cast<const float*>(ld + t0 * row_l), n, w_gate,
+                                       w_up, w_down, tables, k_pre, &chunk_opts, yd + t0 * row_x, nullptr, ws, main_bytes,
+                                       cuda_stream);
         t_keep_status = false;
         if (rc != EXFOLD_OK) return rc;
         EXFOLD_CUDA(cudaEventRecord(h.computed[c], s));

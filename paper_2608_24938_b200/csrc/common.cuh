@@ -40,6 +40,8 @@ __device__ __forceinline__ void report_timeout(DeviceStatus* st, int where) {
 
 // host-side launch accounting
 void count_launch(int n = 1);
+// Synchronises the stream, decodes and clears the device status record at `rec`
+int read_status_record(void* rec, cudaStream_t s);
 
 // Programmatic dependent launch: every kernel of the library is launched with the "programmatic stream
 // serialization" attribute, lets its successor be scheduled early (grid_dep_launch) and waits for its

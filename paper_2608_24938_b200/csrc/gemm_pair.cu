@@ -108,9 +108,6 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
         ptx::tmem_relinquish_pair();
     }
     grid_dep_wait();  // everything below reads what the routing kernels (or GEMM-1) wrote
-#ifdef EXFOLD_TRACE_OVERLAP
-    if (threadIdx.x == 0 && MODE == 0) g_trace[2][blockIdx.x][0] = ptx::globaltimer_ns();
-#endif
     const int G = p.G;
     for (int i = threadIdx.x; i <= G; i += kPThreads) s_off[i] = p.offsets[i];
     ptx::tc_fence_before();
@@ -209,10 +206,6 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
             int stage = 0, phase = 0, iter = 0;
             bool ok = true, ready = false;
             static_assert(kPStages == 6, "the k-loop below is written out for six ring stages");
-#ifdef EXFOLD_TRACE
-            int kbt = 0;
-            long long n_polls = 0, n_ready = 0;
-#endif
             for (int w = w_begin; w < total && ok; w += w_stride, ++iter) {
                 const int as = iter & 1, aphase = (iter >> 1) & 1;
                 if (!ptx::mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag, p.status, 2)) break;
@@ -230,7 +223,6 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
             ok = false;                                                                                             \
             break;                                                                                                  \
         }                                                                                                           \
-        EXFOLD_PAIR_TRACE_KB();                                                                                     \
         ready = ptx::umma_kblock_bf16_pair(d_tmem, lo0 + (S) * lo_step, lo0 + (S) * lo_step + lo_b, desc_hi32,    \
                                            idesc, kb > 0 ? 1u : 0u, &empty_bar[S], &full_bar[NS], nphase);          \
         if (NS == 0) phase ^= 1;                                                                                    \
@@ -239,27 +231,6 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
             break;                                                                                                  \
         }                                                                                                           \
     }
-#ifdef EXFOLD_TRACE
-                // the leader of one pair logs when each k-block's (with EXFOLD_TRACE_TILE: item's) operands were ready
-#ifdef EXFOLD_TRACE_TILE
-#define EXFOLD_PAIR_TRACE_COND (kb == 0)
-#else
-#define EXFOLD_PAIR_TRACE_COND true
-#endif
-#define EXFOLD_PAIR_TRACE_KB()                                                                       \
-    do {                                                                                             \
-        n_polls += 1;                                                                                \
-        n_ready += ready ? 1 : 0;                                                                    \
-        if (MODE == EXFOLD_TRACE_KB_MODE && blockIdx.x == 10 && kbt < 1280 && EXFOLD_PAIR_TRACE_COND) { \
-            unsigned long long* flat = &g_trace[3][0][0];                                            \
-            flat[kbt] = (unsigned long long)clock64();                                               \
-            if ((kbt & 15) == 0) flat[1280 + kbt] = ptx::globaltimer_ns();                           \
-            ++kbt;                                                                                   \
-        }                                                                                            \
-    } while (0)
-#else
-#define EXFOLD_PAIR_TRACE_KB() ((void)0)
-#endif
                 while (ok && kb < nkb) {
                     switch (stage) {
                         case 0: EXFOLD_PAIR_KBLOCK(0)
@@ -272,11 +243,8 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
                     if (kb < nkb) stage = 0;  // fell through the last stage: the ring wraps
                 }
 #undef EXFOLD_PAIR_KBLOCK
-#undef EXFOLD_PAIR_TRACE_KB
                 if (ok) ptx::umma_commit_pair(&tfull_bar[as], 3);
             }
-            EXFOLD_TRACE_SET(MODE, 12, n_polls);  // k-blocks issued / of which the next stage was already complete
-            EXFOLD_TRACE_SET(MODE, 13, n_ready);
         }
         __syncwarp();
     } else {
@@ -353,9 +321,6 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
     }
 
     // ------------------------------------------------ teardown
-#ifdef EXFOLD_TRACE_OVERLAP
-    if (threadIdx.x == 0 && MODE == 0) g_trace[2][blockIdx.x][1] = ptx::globaltimer_ns();
-#endif
     if (threadIdx.x == 64) grid_dep_launch();  // after the epilogue loop, as in the one-CTA kernel
     ptx::tc_fence_before();
     __syncthreads();

@@ -19,15 +19,10 @@
 #include "common.cuh"
 #include "ptx.cuh"
 
-#ifndef EXFOLD_TRACE_KB_MODE
-#define EXFOLD_TRACE_KB_MODE 0  // trace builds: which prefill GEMM (0 or 1) logs per-k-block timestamps
-#endif
-
 namespace exfold {
 
 namespace {
 
-constexpr int kTraceKb = 1280;  // trace builds: k-blocks logged (table 3 of the trace array holds 2 x 1280 words)
 constexpr int kBK = kGemmBK;                  // K elements per stage: one swizzle row (128 or 64 bytes)
 #ifndef EXFOLD_STAGES
 #define EXFOLD_STAGES (EXFOLD_BK == 64 ? 4 : 9)
@@ -106,12 +101,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     unsigned char* tiles =
         reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int kTr = MODE;  // trace table of this kernel (debug builds only)
-    (void)kTr;
-    if (threadIdx.x == 0) EXFOLD_TRACE_SET(kTr, 0, ptx::globaltimer_ns());
-    long long tr_wait = 0, tr_wait2 = 0;
-    (void)tr_wait;
-    (void)tr_wait2;
     // ---- prologue that does not depend on earlier kernels: overlaps their tail under programmatic launch
     if (threadIdx.x == 0) {
         ptx::prefetch_tmap(&p.tm_a);
@@ -217,7 +206,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     const int stage_bytes = DEC ? a_bytes + kBTileBytes : kStageBytes;
     const int stages = DEC ? min(kMaxStages, (kStages * kStageBytes - (kATileBytes - a_bytes)) / stage_bytes) : kStages;
     volatile int* abort_flag = &abort_s;
-    if (threadIdx.x == 0) EXFOLD_TRACE_SET(kTr, 1, ptx::globaltimer_ns());
 
     if (warp == 0 || warp >= 6) {
         // ------------------------------------------------ TMA producers (k-block c belongs to producer c % kProducers)
@@ -236,9 +224,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                 const int brow = MODE == 0 ? expert * p.I + it.n_idx * 128 : expert * p.d + it.n_idx * 256;
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (turn == me) {
-                        bool got;
-                        EXFOLD_TRACE_ADD(tr_wait,
-                                         got = ptx::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, p.status, 1));
+                        const bool got = ptx::mbar_wait(&empty_bar[stage], phase ^ 1, abort_flag, p.status, 1);
                         if (!got) {
                             ok = false;
                             break;
@@ -258,8 +244,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                 }
             }
             if (me == 0) {
-                EXFOLD_TRACE_SET(kTr, 3, tr_wait);
-                EXFOLD_TRACE_SET(kTr, 4, ptx::globaltimer_ns());
             }
         }
         __syncwarp();
@@ -268,9 +252,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         if (lane == 0) {
             constexpr uint32_t idesc = ptx::make_idesc_bf16(128, 256);
             int stage = 0, phase = 0, iter = 0;
-#ifdef EXFOLD_TRACE
-            int kbt = 0;
-#endif
             // This one thread's instruction stream paces the tensor pipe (a k-block is 4 MMAs = 512 pipe cycles),
             // so the loop carries as little as possible: the descriptors' low words advance by a constant per stage
             // (the high word never changes), and the readiness of the NEXT stage is polled before this stage's MMAs
@@ -283,35 +264,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
             bool ready = false;
             for (int w = w_begin; w < total && ok; w += w_stride, ++iter) {
                 const int as = iter & 1, aphase = (iter >> 1) & 1;
-                bool got;
-                EXFOLD_TRACE_ADD(tr_wait2, got = ptx::mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag, p.status, 2));
+                const bool got = ptx::mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag, p.status, 2);
                 if (!got) break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + as * 256;
                 const int kpart = ks == 1 ? 0 : w % ks;
                 const int kb0 = kpart * kb_per, kb1 = min(nkb, kb0 + kb_per);
-#ifdef EXFOLD_TRACE
-                // one CTA of the chosen prefill GEMM logs when each k-block's (EXFOLD_TRACE_TILE: work item's) operands
-                // were ready: cycles, and the ns timer with every 16th entry (for the clock rate)
-#ifdef EXFOLD_TRACE_PAIR
-#define EXFOLD_KB_TRACE_COND false
-#elif defined(EXFOLD_TRACE_TILE)
-#define EXFOLD_KB_TRACE_COND (kb == kb0)
-#else
-#define EXFOLD_KB_TRACE_COND true
-#endif
-#define EXFOLD_KB_TRACE()                                                                                     \
-    do {                                                                                                      \
-        if (MODE == EXFOLD_TRACE_KB_MODE && !DEC && blockIdx.x == 5 && kbt < kTraceKb && EXFOLD_KB_TRACE_COND) { \
-            unsigned long long* flat = &g_trace[3][0][0];                                                     \
-            flat[kbt] = (unsigned long long)clock64();                                                        \
-            if ((kbt & 15) == 0) flat[kTraceKb + kbt] = ptx::globaltimer_ns();                                \
-            ++kbt;                                                                                            \
-        }                                                                                                     \
-    } while (0)
-#else
-#define EXFOLD_KB_TRACE() ((void)0)
-#endif
                 if constexpr (!DEC && kStages == 4) {
                     // Prefill: the k-loop is written out once per ring stage (switch into the stage the ring stands
                     // at), so a k-block costs this thread the MMA sequence, one compare and one branch.
@@ -324,7 +282,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
             ok = false;                                                                                              \
             break;                                                                                                   \
         }                                                                                                            \
-        EXFOLD_KB_TRACE();                                                                                           \
         constexpr uint32_t step = (uint32_t)kStageBytes >> 4, off_b = (uint32_t)kATileBytes >> 4;                    \
         ready = ptx::umma_kblock_bf16(d_tmem, lo0 + (S) * step, lo0 + (S) * step + off_b, desc_hi32, idesc,         \
                                       kb > kb0 ? 1u : 0u, &empty_bar[S], &full_bar[NS], nphase);                     \
@@ -347,14 +304,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                 } else {
                     for (int kb = kb0; kb < kb1; ++kb) {
                         if (!ready) {
-                            EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3));
-                            if (!got) {
+                            if (!ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3)) {
                                 ok = false;
                                 break;
                             }
                         }
-                        if (iter == 0 && kb == kb0) EXFOLD_TRACE_SET(kTr, 9, ptx::globaltimer_ns());
-                        EXFOLD_KB_TRACE();
                         const int ns = stage + 1 == stages ? 0 : stage + 1;
                         const int nphase = ns == 0 ? phase ^ 1 : phase;
                         ready = ptx::umma_kblock_bf16(d_tmem, a_lo, a_lo + lo_b, desc_hi32, idesc, kb > kb0 ? 1u : 0u,
@@ -364,13 +318,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                         phase = nphase;
                     }
                 }
-#undef EXFOLD_KB_TRACE
                 if (ok) ptx::umma_commit(&tfull_bar[as]);
             }
-            EXFOLD_TRACE_SET(kTr, 5, tr_wait);
-            EXFOLD_TRACE_SET(kTr, 6, tr_wait2);
-            EXFOLD_TRACE_SET(kTr, 7, ptx::globaltimer_ns());
-            EXFOLD_TRACE_SET(kTr, 10, iter);
         }
         __syncwarp();
     } else {
@@ -383,8 +332,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
             // lane 0 waits; the warp takes one decision, so the warp-wide TMEM loads below stay convergent
             int ok = 1;
             if (lane == 0) {
-                bool got;
-                EXFOLD_TRACE_ADD(tr_wait, got = ptx::mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status, 4));
+                const bool got = ptx::mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status, 4);
                 ok = got ? 1 : 0;
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -478,8 +426,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     // One thread fires it, after the epilogue loop (a single call marks the whole CTA as triggered).
     if (threadIdx.x == 64) {
         grid_dep_launch();
-        EXFOLD_TRACE_SET(kTr, 8, tr_wait);
-        EXFOLD_TRACE_SET(kTr, 11, ptx::globaltimer_ns());
     }
     ptx::tc_fence_before();
     __syncthreads();
@@ -488,7 +434,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
-    if (threadIdx.x == 0) EXFOLD_TRACE_SET(kTr, 2, ptx::globaltimer_ns());
 }
 
 }  // namespace

@@ -51,3 +51,17 @@ extern "C" int exfold_moe_decode_noalloc(const exfold_layer* layer, const void* 
                                (size_t)EXFOLD_STATIC_SCRATCH_BYTES, cuda_stream);
     return rc == EXFOLD_ERR_WORKSPACE_TOO_SMALL ? EXFOLD_ERR_EXCEEDS_STATIC_SCRATCH : rc;
 }
+
+// The status record of the calls above lives at the start of the built-in array, where the caller cannot
+// point exfold_device_status at it; this is the same check for that record.
+extern "C" int exfold_device_status_noalloc(void* cuda_stream) {
+    void* ws = scratch_for_current_device();
+    if (ws == nullptr) return EXFOLD_ERR_CUDA;
+    return exfold::read_status_record(ws, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int exfold_static_scratch_address(void** address) {
+    if (address == nullptr) return EXFOLD_ERR_INVALID_ARG;
+    *address = scratch_for_current_device();
+    return *address != nullptr ? EXFOLD_OK : EXFOLD_ERR_CUDA;
+}

@@ -323,24 +323,4 @@ __device__ __forceinline__ void red_add_f32(float* gptr, float a) {
 
 }  // namespace ptx
 
-// ------------------------------------------------------------------ optional tracing (debug builds only)
-// With -DEXFOLD_TRACE every tensor-core kernel records, per CTA, a few timestamps and the cycles
-// each role spent waiting; exfold_debug_read_trace() copies them out. Compiled out otherwise.
-#ifdef EXFOLD_TRACE
-constexpr int kTraceSlots = 16;
-extern __device__ unsigned long long g_trace[4][kMaxCtas][kTraceSlots];  // [kernel][cta][slot]
-#define EXFOLD_TRACE_SET(kern, slot, val) (g_trace[kern][blockIdx.x][slot] = (unsigned long long)(val))
-#define EXFOLD_TRACE_ADD(var, expr)                  \
-    do {                                             \
-        long long t__ = clock64();                   \
-        expr;                                        \
-        var += clock64() - t__;                      \
-    } while (0)
-#else
-#define EXFOLD_TRACE_SET(kern, slot, val) ((void)0)
-#define EXFOLD_TRACE_ADD(var, expr) \
-    do {                            \
-        expr;                       \
-    } while (0)
-#endif
 }  // namespace exfold

@@ -3,9 +3,10 @@
 // CTA. The kernel runs as one cluster of 8 CTAs, each holding a full copy of that state: the per-token
 // Top-K (instruction-issue bound on a single SM), the target search (each CTA keeps its slice of the
 // loss / scalar table rows in shared memory) and the row lists are dealt over the CTAs and their results
-// broadcast into every copy through distributed shared memory; the cheap steps in between are replicated. Also builds the execution lists for the weight-streaming FFN: rows sorted
-// by pool rank, duplicate (token, expert) slots merged ("routes folded into the same target
-// are coalesced before expert computation").
+// broadcast into every copy through distributed shared memory; the cheap steps in between are replicated.
+// Also builds the execution lists for the weight-streaming FFN: rows sorted by pool rank, duplicate
+// (token, expert) slots merged so that each pool expert runs once per token (Method, "Unified Expert
+// Folding", the remark after Eq. 4).
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -16,12 +17,6 @@ namespace exfold {
 namespace {
 
 namespace cg = cooperative_groups;
-
-#ifdef EXFOLD_TRACE
-#define DEC_T(slot) if (threadIdx.x == 0 && blockIdx.x == 0) g_trace[2][0][slot] = ptx::globaltimer_ns()
-#else
-#define DEC_T(slot) ((void)0)
-#endif
 
 constexpr int kDecThreads = 1024;
 constexpr int kDecMaxSlots = 4096;
@@ -68,10 +63,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     const int s_lo = min(N, rank * rows_per), s_hi = min(N, s_lo + rows_per);
     float* tL = reinterpret_cast<float*>(smraw + kDecSmemBytes);
     float* tS = tL + (size_t)rows_per * N;
-    DEC_T(0);
     grid_dep_launch();
     grid_dep_wait();
-    DEC_T(1);
     if (p.status != nullptr && rank == 0 && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
     for (int e = threadIdx.x; e < N; e += kDecThreads) {
         sm.acc[e] = 0ull;
@@ -162,7 +155,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     if (!cleared) cluster.barrier_wait();  // warps without a token
     asm volatile("cp.async.wait_all;" ::: "memory");
     cluster.sync();  // all routes and sums have landed in every copy; this CTA's table rows are in place
-    DEC_T(2);
 
     const int nslots = B * K;
     if (is_static) {
@@ -185,7 +177,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         for (int e = threadIdx.x; e < N; e += kDecThreads)
             sm.score[e] = (double)sm.acc[e] * (1.0 / 9007199254740992.0) * (double)sm.hh[e];
     __syncthreads();
-    DEC_T(3);
     // pool = best min(M, |U|) experts of the union by (score desc, id asc): rank by counting. Experts are
     // dealt round-robin over the CTAs, one warp per expert; ranks are broadcast to every copy.
     if (!is_static) {
@@ -212,7 +203,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
     } else {
         __syncthreads();
     }
-    DEC_T(4);
     const int P = sm.P;
     // ---- Eq. 12 for the source experts of this CTA's slice (one warp per source, table rows in shared
     // memory): itself if in the pool, else its min-loss pool expert; the result goes to every copy.
@@ -243,7 +233,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         }
         cluster.sync();  // targets of all slices are in every copy
     }
-    DEC_T(5);
     // ---- Eq. 14: remap every slot in place (each CTA on its own copy); [B][K] layout kept
     for (int s = threadIdx.x; s < nslots; s += kDecThreads) {
         int e = sm.ids[s];
@@ -273,7 +262,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         if (threadIdx.x == 0) *p.pool_size = P;
     }
     __syncthreads();
-    DEC_T(6);
     // ---- execution lists: one row per distinct (token, pool expert), grouped by pool rank. Groups are
     // dealt round-robin over the cluster's CTAs; pass 0 counts and broadcasts, pass 1 writes the rows.
     for (int pass = 0; pass < 2; ++pass) {
@@ -324,7 +312,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
             __syncthreads();
         }
     }
-    DEC_T(7);
     if (rank != 0) return;
     const int G = P + (p.n_shared ? 1 : 0);
     for (int g = threadIdx.x; g <= G; g += kDecThreads) {
@@ -348,7 +335,6 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
         p.n_groups[0] = G;
         p.n_groups[1] = sm.goff[G];  // total rows
     }
-    DEC_T(8);
 }
 
 

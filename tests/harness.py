@@ -51,7 +51,7 @@ class Case:
         return [t.numpy() for t in self.tables_host]
 
     # ---------------------------------------------------------------- GPU runs
-    def run_prefill(self, Kp, with_meta=True):
+    def run_prefill(self, Kp, with_meta=True, gemm_path=0):
         ex, cfg, T = self.ex, self.cfg, self.T
         K, N = cfg.top_k, cfg.n_experts
         ws = self.workspace(T, Kp)
@@ -63,8 +63,12 @@ class Case:
                         w=torch.full((T, Kp), float("nan"), dtype=torch.float32, device=self.dev),
                         omit_src=torch.full((T, K - Kp), -7, **i32), omit_tgt=torch.full((T, K - Kp), -7, **i32),
                         perm=torch.full((T * Kp,), -7, **i32), offsets=torch.full((N + 1,), -7, **i32))
-        ex.exfold_moe_prefill(self.layer, self.d_x, self.d_lg, self.d_wg, self.d_wu, self.d_wd, self.tables, Kp, y, ws,
-                              meta=meta)
+        if gemm_path:
+            ex.exfold_moe_prefill_ex(self.layer, self.d_x, self.d_lg, self.d_wg, self.d_wu, self.d_wd, self.tables, Kp, y,
+                                     ws, gemm_path=gemm_path, meta=meta)
+        else:
+            ex.exfold_moe_prefill(self.layer, self.d_x, self.d_lg, self.d_wg, self.d_wu, self.d_wd, self.tables, Kp, y,
+                                  ws, meta=meta)
         assert ex.exfold_device_status(ws) == 0
         out = {k: v.cpu().numpy() for k, v in (meta or {}).items()}
         out["y"] = y.float().cpu().numpy()

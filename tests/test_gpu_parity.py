@@ -219,9 +219,9 @@ def test_bf16_several_tiles_and_ragged_tail():
 
 
 @pytest.mark.parametrize("shape", ["skewed", "shared", "top1"])
-def test_prefill_on_cta_pairs_matches_oracle_and_the_one_cta_kernel(shape, monkeypatch):
-    """EXFOLD_PAIR_GEMM=2 runs every pair of row tiles of a group on the CTA-pair kernel and the odd last tiles on the
-    one-CTA kernel, whatever the size; =0 keeps everything on the one-CTA kernel. Both must match the oracle, and
+def test_prefill_on_cta_pairs_matches_oracle_and_the_one_cta_kernel(shape):
+    """gemm_path = 2 runs every pair of row tiles of a group on the CTA-pair kernel and the odd last tiles on the
+    one-CTA kernel, whatever the size; = 1 keeps everything on the one-CTA kernel. Both must match the oracle, and
     each other to the last bit (the same products are accumulated in the same order)."""
     if shape == "skewed":    # groups of 0, 1, 2, 3, ... row tiles, ragged last tiles, K and N tails
         cfg = small_bf16(n_experts=8, hidden=512, inter=832, top_k=2, prefill_tokens=1500, logits="zipf", zipf_s=1.5)
@@ -235,11 +235,8 @@ def test_prefill_on_cta_pairs_matches_oracle_and_the_one_cta_kernel(shape, monke
     case = Case(cfg)
     for Kp in Kps:
         ref = case.oracle_prefill(Kp)
-        monkeypatch.setenv("EXFOLD_PAIR_GEMM", "2")
-        got_pair = case.run_prefill(Kp)
-        monkeypatch.setenv("EXFOLD_PAIR_GEMM", "0")
-        got_one = case.run_prefill(Kp)
-        monkeypatch.delenv("EXFOLD_PAIR_GEMM")
+        got_pair = case.run_prefill(Kp, gemm_path=2)
+        got_one = case.run_prefill(Kp, gemm_path=1)
         counts = np.diff(ref["offsets"])
         assert counts.max() >= 256          # at least one whole pair of row tiles
         check_prefill_meta(got_pair, ref)
