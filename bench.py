@@ -1,8 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the folded-MoE layer (ExFold hot path) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mixtral|qwen3|glm45air|tiny]
-                    [--k-pre K'] [--pool-m M] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload glm45air|mixtral|qwen3|tiny] [--k-pre K'] [--pool-m M] ...
 
 One step = one pass of the whole hot path: a prefill call over T tokens (token-level Top-K'
 folding) followed by a decode call over a batch of B tokens (pool-M folding), on seeded
@@ -12,7 +12,13 @@ synthetic inputs shaped like the named model. Prints ONE JSON line (rank 0):
   e2e          the same metric through the host-buffer entry points (pinned host x/logits in, y out)
   roofline     dominant prefill kernel (grouped GEMM-1) against the measured bf16 tensor peak
   cpu_baseline the CPU oracle timed on this machine's host cores on a bounded sample (rank 0, N=1)
-With N > 1 (torchrun) every rank runs an independent replica of the layer: the path has no
+  sustained    the headline prefill call back to back for >= 2 s against the sustained bf16 peak
+  configs      the same measurements for every other benchmark configuration (N=1, no --workload):
+               Mixtral-shaped, Qwen3-shaped (K' = 4 and 6, M = 16/32/64), tiny fp32, and the
+               batch x pool decode sweep on the Qwen3 shape
+Without --workload the headline is the largest single-GPU configuration (GLM-4.5-Air-shaped) and
+`configs` carries the rest; with --workload only that layer is measured (profiling, reduced cases).
+With N > 1 (torchrun) every rank runs an independent replica of the headline layer: the path has no
 exchange step, so there is no collective on the data path.
 --impl reference times the CPU oracle alone (there is no reference implementation to install).
 """
@@ -33,11 +39,17 @@ if ROOT not in sys.path:
 
 import synth_inputs as si  # noqa: E402
 
+HEADLINE = "glm45air"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}  # the figures the benchmark spec names
 # DRAM bytes measured by ncu (dram__bytes_read.sum + dram__bytes_write.sum) divided by the algorithmic
-# bytes of the same launch, from the reduced-case ncu captures whose summaries are under profiles/.
-# Traffic grows with the weights, so the full-size figure is this ratio times the full-size algorithmic bytes.
-NCU_TRAFFIC_RATIO = {"gemm1": 511.3 / 502.3, "decode_gateup": 239.3 / 234.9}
+# bytes of the same launch, from the reduced-case ncu captures whose summaries are under profiles/
+# (same rows per expert as the full-size workload, fewer experts or a shorter intermediate size so that
+# the capture stays small). Traffic grows with the weights, so the full-size figure is this ratio times
+# the full-size algorithmic bytes. A shape without a capture reports traffic = null.
+NCU_TRAFFIC_RATIO = {
+    "mixtral": {"gemm1": 511.3 / 502.3, "decode_gateup": 239.3 / 234.9},
+}
 
 
 def log(*a):
@@ -90,6 +102,11 @@ class ClockSampler(threading.Thread):
                 pass
             time.sleep(self.period)
 
+    def finish(self):
+        self.stop_flag.set()
+        self.join()
+        return self.summary()
+
     def summary(self):
         if not self.ok or not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "note": "no NVML samples"}
@@ -103,12 +120,12 @@ def build_inputs(cfg, T, B):
                lgd=si.router_logits(cfg, B, "logits_dec"))
     inp["wg"], inp["wu"], inp["wd"] = si.expert_weights(cfg)
     inp["tables"] = si.synthetic_tables(cfg)
-    log(f"[bench] inputs generated in {time.time() - t0:.1f}s")
+    log(f"[bench] {cfg.name}: inputs generated in {time.time() - t0:.1f}s")
     return inp
 
 
-def oracle_sample_run(cfg, inp, Kp, M, n_tokens, seed=7):
-    """CPU oracle on a seeded sample of prefill tokens (routing at full size) and on the full decode batch."""
+def oracle_sample_run(cfg, inp, Kp, n_tokens, seed=7):
+    """CPU oracle on a seeded sample of prefill tokens (routing at full size)."""
     import oracle
     A = si.as_oracle_array
     S, L, h, lnh = [t.numpy() for t in inp["tables"]]
@@ -157,8 +174,15 @@ def rel_err(y, ref):
     return float(np.abs(y - ref).max() / np.abs(ref).max()), float(np.linalg.norm(y - ref) / np.linalg.norm(ref))
 
 
-def workload_config(args):
-    cfg = si.CONFIGS[args.workload]
+def r4(v):
+    """Round to 5 significant digits (keeps the JSON line short)."""
+    if v is None:
+        return None
+    return float(f"{float(v):.5g}")
+
+
+def workload_config(args, name=None):
+    cfg = si.CONFIGS[name or args.workload or HEADLINE]
     over = {}
     if args.tokens:
         over["prefill_tokens"] = args.tokens
@@ -166,35 +190,298 @@ def workload_config(args):
         over["decode_batch"] = args.batch
     if args.inter:
         over["inter"] = args.inter
+    if args.experts:
+        over["n_experts"] = args.experts
     if over:
         cfg = si.scaled(cfg, name=cfg.name + "-reduced", **over)
     return cfg
 
 
-def stack_leg(ex, cfg, layer, tables, weights, xd, M, L, dev, flush, reps=10):
-    """L decode layers of the workload's shape, each = router scores (W_r x) + folded decode layer, one after the
-    other on one stream. Every layer owns its weights (device copies rolled along the expert axis, so no weight
-    line is reused between layers) and its router matrix; all layers read the same x (the layers are sequential
-    in time, independent in data). Timed as plain stream launches and as one captured CUDA graph."""
+class Flush:
+    """Evicts L2 between calls by READING a 512 MiB buffer: the cache is left full of clean lines.
+    (Writing the buffer instead would leave ~126 MB of dirty lines whose write-back is then charged to
+    the first reads of the timed kernel: about 20 us of foreign DRAM traffic per call.)"""
+
+    def __init__(self, dev):
+        import torch
+        self.torch = torch
+        self.buf = torch.zeros(128 << 20, dtype=torch.int32, device=dev)  # 512 MiB, > 4x L2
+
+    def __call__(self):
+        self.torch.sum(self.buf)
+
+
+class Workload:
+    """One synthetic layer resident on the device, with the calls the benchmark times."""
+
+    def __init__(self, ex, cfg, dev, batches=None):
+        import torch
+        self.ex, self.cfg, self.dev, self.torch = ex, cfg, dev, torch
+        self.T, self.B = cfg.prefill_tokens, cfg.decode_batch
+        maxB = max([self.B] + list(batches or []))
+        self.inp = build_inputs(cfg, self.T, maxB)
+        g = lambda t: t.to(dev)
+        inp = self.inp
+        self.x, self.lg = g(inp["x"]), g(inp["lg"])
+        self.xd_all, self.lgd_all = g(inp["xd"]), g(inp["lgd"])
+        self.wg, self.wu, self.wd = g(inp["wg"]), g(inp["wu"]), g(inp["wd"])
+        self.tabs = [g(t) for t in inp["tables"]]
+        self.tables = ex.make_tables(*self.tabs)
+        self.layer = ex.make_layer(cfg.n_experts, cfg.n_shared, cfg.hidden, cfg.inter, cfg.top_k, cfg.dtype)
+        self.ws = ex.alloc_workspace(self.layer, max(self.T, maxB), cfg.top_k, host_staging=True)
+        self.y = torch.empty((self.T, cfg.hidden), dtype=self.wg.dtype, device=dev)
+        self.el = 2 if cfg.dtype == "bf16" else 4
+        self.set_batch(self.B)
+
+    def set_batch(self, B):
+        torch = self.torch
+        self.B = B
+        self.xd, self.lgd = self.xd_all[:B].contiguous(), self.lgd_all[:B].contiguous()
+        self.yd = torch.empty((B, self.cfg.hidden), dtype=self.wg.dtype, device=self.dev)
+        self.dmeta = dict(pool_size=torch.zeros(1, dtype=torch.int32, device=self.dev))
+
+    def prefill(self, Kp, meta=None):
+        self.ex.exfold_moe_prefill(self.layer, self.x, self.lg, self.wg, self.wu, self.wd, self.tables, Kp, self.y,
+                                   self.ws, meta=meta)
+
+    def decode(self, M):
+        self.ex.exfold_moe_decode(self.layer, self.xd, self.lgd, self.wg, self.wu, self.wd, self.tables, M, self.yd,
+                                  self.ws, meta=self.dmeta)
+
+    def status_ok(self, what):
+        assert self.ex.exfold_device_status(self.ws) == 0, f"device status after {what}"
+
+    def timed(self, fn, steps, warmup, flush):
+        """Per-call CUDA events on the launching stream, L2 evicted before every call. Returns ms per call."""
+        torch = self.torch
+        for _ in range(warmup):
+            flush()
+            fn()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in ev:
+            flush()
+            a.record()
+            fn()
+            b.record()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in ev]
+
+    def kernel_times(self, fn, reps, flush):
+        ex, torch = self.ex, self.torch
+        ex.exfold_profile_enable(True)
+        kern = {}
+        for _ in range(reps):
+            flush()
+            fn()
+            torch.cuda.synchronize()
+            for k_, v in ex.exfold_profile_read().items():
+                kern.setdefault(k_, []).append(v)
+        ex.exfold_profile_enable(False)
+        return {k_: float(np.mean(v)) for k_, v in kern.items()}
+
+    def free(self):
+        for k in list(self.__dict__):
+            if k not in ("torch",):
+                self.__dict__.pop(k)
+        self.torch.cuda.empty_cache()
+
+
+def prefill_report(wl, Kp, ms_list, kern, peaks, peak_src, world=1):
+    """Fractions for one prefill configuration. Algorithmic work: 6 d I flop per (token, executed expert);
+    compulsory HBM bytes: every touched expert's weights once + x + y + logits."""
     import torch
-    wg, wu, wd = weights
-    B, N, d = xd.shape[0], cfg.n_experts, cfg.hidden
-    per = [(torch.roll(wg, l, 0), torch.roll(wu, l, 0), torch.roll(wd, l, 0)) if l else (wg, wu, wd) for l in range(L)]
-    wr0 = si.router_weights(cfg).to(dev)
+    cfg = wl.cfg
+    T, N, d, I, el = wl.T, cfg.n_experts, cfg.hidden, cfg.inter, wl.el
+    ms = float(np.mean(ms_list))
+    rows = T * Kp + T * cfg.n_shared
+    flop = rows * 6.0 * d * I
+    off = torch.zeros(N + 1, dtype=torch.int32, device=wl.dev)
+    wl.prefill(Kp, meta=dict(offsets=off))
+    torch.cuda.synchronize()
+    touched = int((np.diff(off.cpu().numpy()) > 0).sum()) + cfg.n_shared
+    byts = touched * 3.0 * d * I * el + 2.0 * T * d * el + 4.0 * T * N
+    t_c, t_m = flop / (peaks["bf16_tflops"] * 1e12) * 1e3, byts / (peaks["hbm_gbs"] * 1e9) * 1e3
+    out = {"k_pre": Kp, "ms": r4(ms), "ms_min": r4(np.min(ms_list)), "tokens_per_s": r4(world * T / (ms * 1e-3)),
+           "useful_tflops": r4(flop / (ms * 1e-3) / 1e12),
+           "frac_of_bf16_peak": r4(flop / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]),
+           "frac_of_bf16_sustained": r4(flop / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]),
+           "frac_of_nominal_bf16": r4(flop / (ms * 1e-3) / 1e12 / NOMINAL["bf16_tflops"]),
+           "touched_experts": touched, "t_compute_ms": r4(t_c), "t_hbm_ms": r4(t_m),
+           "frac_of_bound": r4(max(t_c, t_m) / ms), "flop": flop, "compulsory_bytes": byts}
+    if kern:
+        out["kernels_ms"] = {k: r4(v) for k, v in kern.items()}
+        if "gemm1_gateup_swiglu" in kern:
+            f1, f2 = rows * 4.0 * d * I, rows * 2.0 * d * I
+            out["gemm1_frac"] = r4(f1 / (kern["gemm1_gateup_swiglu"] * 1e-3) / 1e12 / peaks["bf16_tflops"])
+            out["gemm2_frac"] = r4(f2 / (kern["gemm2_down_combine"] * 1e-3) / 1e12 / peaks["bf16_tflops"])
+            out["non_gemm_ms"] = r4(sum(v for k, v in kern.items() if k in ("prefill_route", "prefill_scatter",
+                                                                            "convert_bf16")))
+    return out
+
+
+def prefill_roofline(wl, Kp, kern, peaks, peak_src, touched):
+    cfg = wl.cfg
+    T, d, I, el = wl.T, cfg.hidden, cfg.inter, wl.el
+    rows = T * Kp + T * cfg.n_shared
+    if "gemm1_gateup_swiglu" in kern:
+        f1 = rows * 4.0 * d * I
+        ach = f1 / (kern["gemm1_gateup_swiglu"] * 1e-3) / 1e12
+        b1 = touched * 2.0 * d * I * el + rows * d * el + rows * I * el
+        ratio = NCU_TRAFFIC_RATIO.get(cfg.name.replace("-reduced", ""), {}).get("gemm1")
+        return {"kernel": "grouped GEMM-1 (gate/up + SwiGLU), tcgen05", "bound": "tensor", "achieved": r4(ach),
+                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": r4(ach / peaks["bf16_tflops"]),
+                "traffic": None if ratio is None else b1 * ratio,
+                "traffic_note": "ncu reduced-case DRAM bytes / algorithmic bytes x full-size algorithmic bytes"
+                                if ratio else "no ncu capture of this shape",
+                "peak_source": f"{peak_src} burst bf16 matmul", "launch_ms": r4(kern["gemm1_gateup_swiglu"]),
+                "flop_per_launch": f1, "algorithmic_bytes_per_launch": b1}
+    if "simt_ffn" in kern:
+        flop = rows * 6.0 * d * I
+        ach = flop / (kern["simt_ffn"] * 1e-3) / 1e12
+        return {"kernel": "SIMT fp32 expert FFN", "bound": "alu", "achieved": r4(ach), "peak": 72.0,
+                "unit": "TFLOP/s", "frac": r4(ach / 72.0), "traffic": None, "launch_ms": r4(kern["simt_ffn"]),
+                "flop_per_launch": flop, "peak_source": "148 SMs x 128 fp32 lanes x 2 flop x 1.9 GHz"}
+    return None
+
+
+def decode_report(wl, M, ms_list, kern, peaks, static_ms=None):
+    cfg = wl.cfg
+    d, I, el = cfg.hidden, cfg.inter, wl.el
+    ms = float(np.mean(ms_list))
+    pool = int(wl.dmeta["pool_size"].item())
+    byts = (pool + cfg.n_shared) * 3.0 * d * I * el
+    gbs = byts / (ms * 1e-3) / 1e9
+    out = {"batch": wl.B, "pool_m": M, "effective_pool": pool, "us_per_layer": r4(ms * 1e3),
+           "us_min": r4(np.min(ms_list) * 1e3), "pool_weight_bytes": byts, "gbs_on_pool_bytes": r4(gbs),
+           "frac_of_measured_hbm": r4(gbs / peaks["hbm_gbs"]), "frac_of_8tbs": r4(gbs / NOMINAL["hbm_gbs"])}
+    if static_ms is not None:
+        out["static_pool_us_per_layer"] = r4(float(np.mean(static_ms)) * 1e3)
+    if kern:
+        out["kernels_ms"] = {k: r4(v) for k, v in kern.items()}
+    return out
+
+
+def decode_roofline(wl, kern, peaks, pool):
+    cfg = wl.cfg
+    byts = (pool + cfg.n_shared) * 3.0 * cfg.hidden * cfg.inter * wl.el
+    name = cfg.name.replace("-reduced", "")
+    if "decode_ffn" in kern:  # one fused kernel streams gate, up and down weights
+        t = kern["decode_ffn"] * 1e-3
+        ratio = NCU_TRAFFIC_RATIO.get(name, {}).get("decode_ffn")
+        return {"kernel": "decode fused expert FFN (gate/up/down weight stream over the pool), tcgen05", "bound": "hbm",
+                "achieved": r4(byts / t / 1e9), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": r4(byts / t / 1e9 / peaks["hbm_gbs"]), "traffic": None if ratio is None else byts * ratio,
+                "bytes_per_launch": byts, "launch_ms": r4(kern["decode_ffn"])}
+    if "decode_gateup" in kern:
+        gu = byts * 2.0 / 3.0
+        tg = kern["decode_gateup"] * 1e-3
+        ratio = NCU_TRAFFIC_RATIO.get(name, {}).get("decode_gateup")
+        out = {"kernel": "decode GEMM-1 (gate/up weight stream over the pool), tcgen05", "bound": "hbm",
+               "achieved": r4(gu / tg / 1e9), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+               "frac": r4(gu / tg / 1e9 / peaks["hbm_gbs"]), "traffic": None if ratio is None else gu * ratio,
+               "bytes_per_launch": gu, "launch_ms": r4(kern["decode_gateup"])}
+        td = kern.get("decode_down", 0.0) * 1e-3
+        if td > 0:
+            out["down_gbs"] = r4(byts / 3.0 / td / 1e9)
+            out["ffn_gbs"] = r4(byts / (tg + td) / 1e9)
+        return out
+    return None
+
+
+def e2e_leg(wl, Kp, M, reps, flush, world=1):
+    """Through the host-buffer entry points: pinned host x / logits in, y out, copies inside the timed region."""
+    torch, ex, cfg = wl.torch, wl.ex, wl.cfg
+    inp, T, B, d, N = wl.inp, wl.T, wl.B, cfg.hidden, cfg.n_experts
+    xh, lh = inp["x"].pin_memory(), inp["lg"].pin_memory()
+    xdh, ldh = inp["xd"][:B].contiguous().pin_memory(), inp["lgd"][:B].contiguous().pin_memory()
+    yh = torch.empty((T, d), dtype=wl.wg.dtype).pin_memory()
+    ydh = torch.empty((B, d), dtype=wl.wg.dtype).pin_memory()
+    ee = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(reps)]
+    for it in range(reps + 2):
+        k = max(it - 2, 0)
+        flush()
+        ee[k][0].record()
+        ex.exfold_moe_prefill_host(wl.layer, xh, lh, wl.wg, wl.wu, wl.wd, wl.tables, Kp, yh, wl.ws)
+        ee[k][1].record()
+        flush()
+        ee[k][2].record()
+        ex.exfold_moe_decode_host(wl.layer, xdh, ldh, wl.wg, wl.wu, wl.wd, wl.tables, M, ydh, wl.ws)
+        ee[k][3].record()
+        torch.cuda.synchronize()
+    pre = float(np.mean([e[0].elapsed_time(e[1]) for e in ee]))
+    dec = float(np.mean([e[2].elapsed_time(e[3]) for e in ee]))
+    pre, dec = max_over_ranks([pre, dec], world, wl.dev)
+    el = wl.el
+    return {"value": r4(job_tokens_per_s(T, world, pre)), "unit": "tokens/s",
+            "h2d_bytes_per_step": int(T * d * el + T * N * 4 + B * d * el + B * N * 4),
+            "d2h_bytes_per_step": int(T * d * el + B * d * el), "prefill_ms": r4(pre), "decode_us": r4(dec * 1e3)}
+
+
+def cpu_baseline_leg(wl, Kp, M, flop_budget):
+    """The oracle as it stands on a bounded sample of the same workload; the sample doubles as a parity check
+    of the benchmarked outputs (wl.y / wl.yd must hold the results of prefill(Kp) / decode(M))."""
+    import oracle
+    cfg = wl.cfg
+    d, I, K = cfg.hidden, cfg.inter, cfg.top_k
+    per_tok = (Kp + cfg.n_shared) * 6.0 * d * I
+    n_s = int(max(1, min(256, flop_budget / per_tok)))
+    t0 = time.time()
+    o = oracle_sample_run(cfg, wl.inp, Kp, n_s)
+    yg = wl.y.float().cpu().numpy()[o["idx"]]
+    emax, efro = rel_err(yg, o["y"])
+    base = {"value": r4(o["tokens_per_s"]), "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{o['tokens']} seeded prefill tokens (all their routes) of the same workload; routing at "
+                      f"full size; {o['seconds']:.1f}s"}
+    parity = {"prefill_max_err_rel": r4(emax), "prefill_fro_err_rel": r4(efro), "tokens": int(o["tokens"])}
+    if wl.B * (K + cfg.n_shared) * 6.0 * d * I <= 4 * flop_budget:
+        inp = dict(wl.inp)
+        inp["xd"], inp["lgd"] = wl.inp["xd"][:wl.B], wl.inp["lgd"][:wl.B]
+        od = oracle_decode_run(cfg, inp, M)
+        dmax, dfro = rel_err(wl.yd.float().cpu().numpy(), od["y"])
+        base["decode_us_per_layer"] = r4(od["seconds"] * 1e6)
+        parity.update({"decode_max_err_rel": r4(dmax), "decode_fro_err_rel": r4(dfro)})
+    log(f"[bench] {cfg.name}: cpu baseline took {time.time() - t0:.1f}s")
+    return base, parity
+
+
+def static_pool_for(wl, M):
+    torch, ex, cfg = wl.torch, wl.ex, wl.cfg
+    i32 = dict(dtype=torch.int32, device=wl.dev)
+    keep = (torch.empty(M, **i32), torch.empty(cfg.n_experts, **i32),
+            torch.empty(cfg.n_experts, dtype=torch.float32, device=wl.dev))
+    sp = ex.exfold_static_pool_build(wl.layer, wl.tables, M, *keep)
+    return sp, keep
+
+
+def stack_leg(wl, M, L, flush, Kp=None, reps=8):
+    """L layers of the workload's shape run one after the other on one stream, each = router scores (W_r x) + folded
+    layer, every layer with its own weights (device views rolled along the expert axis, so no weight line is reused
+    between layers) and router matrix, layer l+1 reading layer l's output. Timed as plain stream launches and as one
+    captured CUDA graph. Kp = None: decode layers on the decode batch; else prefill layers on the prefill tokens."""
+    torch, ex, cfg = wl.torch, wl.ex, wl.cfg
+    N, d = cfg.n_experts, cfg.hidden
+    per = [(torch.roll(wl.wg, l, 0), torch.roll(wl.wu, l, 0), torch.roll(wl.wd, l, 0)) if l else (wl.wg, wl.wu, wl.wd)
+           for l in range(L)]
+    wr0 = si.router_weights(cfg).to(wl.dev)
     wrs = [torch.roll(wr0, l, 0) for l in range(L)]
-    lgs = [torch.empty((B, N), dtype=torch.float32, device=dev) for _ in range(L)]
-    ys = [torch.empty((B, d), dtype=wg.dtype, device=dev) for _ in range(L)]
-    ws = ex.alloc_workspace(layer, B, cfg.top_k)
+    x0 = wl.xd if Kp is None else wl.x
+    n = x0.shape[0]
+    lgs = [torch.empty((n, N), dtype=torch.float32, device=wl.dev) for _ in range(L)]
+    hs = [x0] + [torch.empty((n, d), dtype=wl.wg.dtype, device=wl.dev) for _ in range(L)]
 
     def run_layers():
         for l in range(L):
-            ex.exfold_router_logits(layer, xd, wrs[l], lgs[l], ws)
-            ex.exfold_moe_decode(layer, xd, lgs[l], per[l][0], per[l][1], per[l][2], tables, M, ys[l], ws)
+            if Kp is None:
+                ex.exfold_moe_decode_layer(wl.layer, hs[l], wrs[l], per[l][0], per[l][1], per[l][2], wl.tables, M,
+                                           hs[l + 1], wl.ws, logits_out=lgs[l])
+            else:
+                ex.exfold_moe_prefill_layer(wl.layer, hs[l], wrs[l], per[l][0], per[l][1], per[l][2], wl.tables, Kp,
+                                            hs[l + 1], wl.ws, logits_out=lgs[l])
 
     def timed(fn):
         ts = []
         for it in range(reps + 2):
-            flush.zero_()
+            flush()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             fn()
@@ -204,9 +491,10 @@ def stack_leg(ex, cfg, layer, tables, weights, xd, M, L, dev, flush, reps=10):
                 ts.append(e0.elapsed_time(e1))
         return float(np.median(ts))
 
-    res = {"layers": L, "what": "router GEMM + folded decode layer per layer, own weights per layer, same x"}
-    res["stream_us_per_layer"] = timed(run_layers) * 1e3 / L
-    assert ex.exfold_device_status(ws) == 0, "device status after the layer stack"
+    res = {"layers": L, "mode": "decode" if Kp is None else "prefill",
+           "what": "router scores + folded layer per layer, own weights per layer, each layer reads the previous output"}
+    res["stream_us_per_layer"] = r4(timed(run_layers) * 1e3 / L)
+    wl.status_ok("the layer stack")
     try:
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
@@ -214,11 +502,84 @@ def stack_leg(ex, cfg, layer, tables, weights, xd, M, L, dev, flush, reps=10):
         with torch.cuda.graph(graph, stream=side):
             run_layers()
         torch.cuda.synchronize()
-        res["graph_us_per_layer"] = timed(graph.replay) * 1e3 / L
-        assert ex.exfold_device_status(ws) == 0, "device status after the graph replays"
+        res["graph_us_per_layer"] = r4(timed(graph.replay) * 1e3 / L)
+        wl.status_ok("the graph replays")
     except Exception as e:  # capture is an optional measurement: report, do not lose the benchmark line
         res["graph_error"] = f"{type(e).__name__}: {e}"[:300]
     return res
+
+
+def measure_config(ex, cfg, dev, args, peaks, peak_src, flush, steps, warmup, with_cpu=True, with_e2e=True,
+                   sweep=None, stack_layers=0):
+    """All measurements of one configuration, device-timed at N=1: every K' of the config for prefill, every M for
+    decode (dynamic pool, and the static pool beside it), per-kernel times, fractions, e2e and the CPU baseline of
+    the config's first (K', M)."""
+    torch = __import__("torch")
+    wl = Workload(ex, cfg, dev, batches=sweep[0] if sweep else None)
+    rec = {"workload": describe(cfg), "dtype": cfg.dtype, "prefill": [], "decode": []}
+    for Kp in cfg.k_pre:
+        ms = wl.timed(lambda: wl.prefill(Kp), steps, warmup, flush)
+        kern = wl.kernel_times(lambda: wl.prefill(Kp), min(steps, 6), flush)
+        rep = prefill_report(wl, Kp, ms, kern, peaks, peak_src)
+        if Kp == cfg.k_pre[0]:
+            rec["roofline"] = prefill_roofline(wl, Kp, kern, peaks, peak_src, rep["touched_experts"])
+        rec["prefill"].append(rep)
+    wl.status_ok("prefill")
+    for M in cfg.pool_m:
+        ms = wl.timed(lambda: wl.decode(M), steps, warmup, flush)
+        kern = wl.kernel_times(lambda: wl.decode(M), min(steps, 6), flush)
+        sp, keep = static_pool_for(wl, M)
+        st = wl.timed(lambda: ex.exfold_moe_decode_static(wl.layer, wl.xd, wl.lgd, wl.wg, wl.wu, wl.wd, sp, wl.yd,
+                                                          wl.ws), steps, warmup, flush)
+        wl.decode(M)  # pool_size / yd of the dynamic pool again
+        torch.cuda.synchronize()
+        rep = decode_report(wl, M, ms, kern, peaks, static_ms=st)
+        rl = decode_roofline(wl, kern, peaks, rep["effective_pool"])
+        if rl:
+            rep["roofline"] = rl
+        rec["decode"].append(rep)
+    wl.status_ok("decode")
+    Kp0, M0 = cfg.k_pre[0], cfg.pool_m[0]
+    if with_e2e:
+        rec["e2e"] = e2e_leg(wl, Kp0, M0, min(steps, 6), flush)
+    if with_cpu and not args.skip_cpu_baseline:
+        wl.prefill(Kp0)
+        wl.decode(M0)
+        torch.cuda.synchronize()
+        rec["cpu_baseline"], rec["parity_sample"] = cpu_baseline_leg(wl, Kp0, M0, args.cpu_flop_budget)
+    if stack_layers:
+        rec["stack"] = [stack_leg(wl, M0, stack_layers, flush), stack_leg(wl, M0, stack_layers, flush, Kp=Kp0)]
+    if sweep:
+        rec["decode_sweep"] = decode_sweep(wl, sweep[0], sweep[1], peaks, flush, max(4, steps // 2), warmup)
+    wl.free()
+    return rec
+
+
+def decode_sweep(wl, batches, pools, peaks, flush, steps, warmup):
+    """Decode batch x pool sweep: us/layer, effective pool, GB/s on the pool's weight bytes, speed-up over the
+    unfolded layer (M = N) of the same batch."""
+    cfg = wl.cfg
+    N, K = cfg.n_experts, cfg.top_k
+    table = []
+    for B in [b for b in batches if b * K <= 4096]:
+        wl.set_batch(B)
+        row = {}
+        for M in pools:
+            ms = wl.timed(lambda: wl.decode(M), steps, warmup, flush)
+            row[M] = decode_report(wl, M, ms, None, peaks)
+        for M in pools:
+            r = row[M]
+            table.append({"B": B, "M": M, "P": r["effective_pool"], "us": r["us_per_layer"],
+                          "gbs": r["gbs_on_pool_bytes"], "frac_hbm": r["frac_of_measured_hbm"],
+                          "speedup_vs_unfolded": r4(row[N]["us_per_layer"] / r["us_per_layer"])})
+    wl.status_ok("the decode sweep")
+    return table
+
+
+def describe(cfg):
+    return (f"{cfg.name}-shaped layer: N={cfg.n_experts}+{cfg.n_shared} experts, d={cfg.hidden}, I={cfg.inter}, "
+            f"top-{cfg.top_k} folded to top-{'/'.join(map(str, cfg.k_pre))}, prefill T={cfg.prefill_tokens}; decode "
+            f"B={cfg.decode_batch}, pool M={'/'.join(map(str, cfg.pool_m))}; logits {cfg.logits}")
 
 
 def run_ours(args, rank, world):
@@ -234,49 +595,25 @@ def run_ours(args, rank, world):
     cfg = workload_config(args)
     Kp = args.k_pre or cfg.k_pre[0]
     M = args.pool_m or cfg.pool_m[0]
-    T, B, K, N, d, I = cfg.prefill_tokens, cfg.decode_batch, cfg.top_k, cfg.n_experts, cfg.hidden, cfg.inter
+    K, N, d, I = cfg.top_k, cfg.n_experts, cfg.hidden, cfg.inter
     peaks, peak_src = load_peaks()
-    inp = build_inputs(cfg, T, B)
-    g = lambda t: t.to(dev)
-    x, lg, xd, lgd = g(inp["x"]), g(inp["lg"]), g(inp["xd"]), g(inp["lgd"])
-    wg, wu, wd = g(inp["wg"]), g(inp["wu"]), g(inp["wd"])
-    tabs = [g(t) for t in inp["tables"]]
-    tables = ex.make_tables(*tabs)
-    layer = ex.make_layer(N, cfg.n_shared, d, I, K, cfg.dtype)
-    ws = ex.alloc_workspace(layer, max(T, B), max(Kp, K), host_staging=True)
-    y = torch.empty((T, d), dtype=wg.dtype, device=dev)
-    yd = torch.empty((B, d), dtype=wg.dtype, device=dev)
-    dmeta = dict(pool_size=torch.zeros(1, dtype=torch.int32, device=dev))
-    flush_buf = torch.zeros(128 << 20, dtype=torch.int32, device=dev)  # 512 MiB, > 4x L2
-
-    class _Flush:
-        """Evicts L2 between calls by READING a 512 MiB buffer: the cache is left full of clean lines.
-        (Writing the buffer instead would leave ~126 MB of dirty lines whose write-back is then charged to
-        the first reads of the timed kernel: about 20 us of foreign DRAM traffic per call.)"""
-
-        def zero_(self):
-            torch.sum(flush_buf)
-
-    flush = _Flush()
-
-    def prefill():
-        ex.exfold_moe_prefill(layer, x, lg, wg, wu, wd, tables, Kp, y, ws)
-
-    def decode():
-        ex.exfold_moe_decode(layer, xd, lgd, wg, wu, wd, tables, M, yd, ws, meta=dmeta)
+    warmup = max(args.warmup, 3)
+    wl = Workload(ex, cfg, dev)
+    T, B = wl.T, wl.B
+    flush = Flush(dev)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        flush.zero_()
-        prefill()
-        decode()
+    for _ in range(warmup):
+        flush()
+        wl.prefill(Kp)
+        wl.decode(M)
     torch.cuda.synchronize()
-    assert ex.exfold_device_status(ws) == 0, "device status after warm-up"
-    pool_size = int(dmeta["pool_size"].item())
+    wl.status_ok("warm-up")
+    pool_size = int(wl.dmeta["pool_size"].item())
 
     # ---- timed region: K steps, per-call CUDA events on the launching stream, L2 flushed between calls
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
@@ -286,85 +623,71 @@ def run_ours(args, rank, world):
     launches0 = ex.exfold_launch_count()
     wall0 = time.perf_counter()
     for k in range(args.steps):
-        flush.zero_()
+        flush()
         ev[k][0].record()
-        prefill()
+        wl.prefill(Kp)
         ev[k][1].record()
-        flush.zero_()
+        flush()
         ev[k][2].record()
-        decode()
+        wl.decode(M)
         ev[k][3].record()
     barrier()
     wall = time.perf_counter() - wall0
     launches = ex.exfold_launch_count() - launches0
-    sampler.stop_flag.set()
-    sampler.join()
-    assert ex.exfold_device_status(ws) == 0, "device status after the timed region"
-    pre_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
-    dec_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))
-    pre_min = float(np.min([e[0].elapsed_time(e[1]) for e in ev]))
-    dec_min = float(np.min([e[2].elapsed_time(e[3]) for e in ev]))
-    pre_ms, dec_ms = max_over_ranks([pre_ms, dec_ms], world, dev)
+    clocks = sampler.finish()
+    wl.status_ok("the timed region")
+    pre_list = [e[0].elapsed_time(e[1]) for e in ev]
+    dec_list = [e[2].elapsed_time(e[3]) for e in ev]
+    pre_ms, dec_ms = max_over_ranks([float(np.mean(pre_list)), float(np.mean(dec_list))], world, dev)
+    pre_list = [v * pre_ms / float(np.mean(pre_list)) for v in pre_list]  # scaled to the slowest rank's mean
+    dec_list = [v * dec_ms / float(np.mean(dec_list)) for v in dec_list]
 
     # ---- per-kernel durations (CUDA events recorded by the library around each launch)
-    ex.exfold_profile_enable(True)
-    kern = {}
     nprof = min(args.steps, 10)
-    for _ in range(nprof):
-        flush.zero_()
-        prefill()
-        torch.cuda.synchronize()
-        for k_, v in ex.exfold_profile_read().items():
-            kern.setdefault(k_, []).append(v)
-        flush.zero_()
-        decode()
-        torch.cuda.synchronize()
-        for k_, v in ex.exfold_profile_read().items():
-            kern.setdefault("dec:" + k_ if k_ == "convert_bf16" else k_, []).append(v)
-    ex.exfold_profile_enable(False)
-    kern = {k_: float(np.mean(v)) for k_, v in kern.items()}
+    kern_p = wl.kernel_times(lambda: wl.prefill(Kp), nprof, flush)
+    kern_d = wl.kernel_times(lambda: wl.decode(M), nprof, flush)
+    pre_rep = prefill_report(wl, Kp, pre_list, kern_p, peaks, peak_src, world)
+    wl.decode(M)
+    torch.cuda.synchronize()
+    dec_rep = decode_report(wl, M, dec_list, kern_d, peaks)
+    rl_d = decode_roofline(wl, kern_d, peaks, pool_size)
+    if rl_d:
+        dec_rep["roofline"] = rl_d
+    if world == 1:
+        sp, keep = static_pool_for(wl, M)
+        st = wl.timed(lambda: ex.exfold_moe_decode_static(wl.layer, wl.xd, wl.lgd, wl.wg, wl.wu, wl.wd, sp, wl.yd,
+                                                          wl.ws), min(args.steps, 10), 3, flush)
+        dec_rep["static_pool_us_per_layer"] = r4(float(np.mean(st)) * 1e3)
+
+    # ---- sustained leg: the headline prefill call back to back for >= 2 s (inputs far exceed L2: no flush needed)
+    sustained = None
+    if not args.skip_sustained:
+        n_calls = int(max(10, min(20000, 2.2e3 / pre_ms)))
+        s2 = ClockSampler(local, period=0.01)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s2.start()
+        e0.record()
+        for _ in range(n_calls):
+            wl.prefill(Kp)
+        e1.record()
+        barrier()
+        ck = s2.finish()
+        sus_ms = max_over_ranks([e0.elapsed_time(e1) / n_calls], world, dev)[0]
+        tf = pre_rep["flop"] / (sus_ms * 1e-3) / 1e12
+        sustained = {"calls": n_calls, "seconds": r4(sus_ms * n_calls * 1e-3), "ms_per_call": r4(sus_ms),
+                     "useful_tflops": r4(tf), "frac_of_bf16_sustained": r4(tf / peaks["bf16_tflops_sustained"]),
+                     "frac_of_bf16_peak": r4(tf / peaks["bf16_tflops"]), "clocks": ck}
+        wl.status_ok("the sustained leg")
 
     # ---- end to end through the host-buffer entry points (pinned host memory, copies inside the timed region)
-    xh, lh = inp["x"].pin_memory(), inp["lg"].pin_memory()
-    xdh, ldh = inp["xd"].pin_memory(), inp["lgd"].pin_memory()
-    yh = torch.empty((T, d), dtype=wg.dtype).pin_memory()
-    ydh = torch.empty((B, d), dtype=wg.dtype).pin_memory()
-    ne2e = min(args.steps, 10)
-    ee = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(ne2e)]
-    for it in range(ne2e + 2):
-        k = max(it - 2, 0)
-        flush.zero_()
-        ee[k][0].record()
-        ex.exfold_moe_prefill_host(layer, xh, lh, wg, wu, wd, tables, Kp, yh, ws)
-        ee[k][1].record()
-        flush.zero_()
-        ee[k][2].record()
-        ex.exfold_moe_decode_host(layer, xdh, ldh, wg, wu, wd, tables, M, ydh, ws)
-        ee[k][3].record()
-        torch.cuda.synchronize()
-    e2e_pre = float(np.mean([e[0].elapsed_time(e[1]) for e in ee]))
-    e2e_dec = float(np.mean([e[2].elapsed_time(e[3]) for e in ee]))
-    e2e_pre, e2e_dec = max_over_ranks([e2e_pre, e2e_dec], world, dev)
-    el = 2 if cfg.dtype == "bf16" else 4
-    h2d = T * d * el + T * N * 4 + B * d * el + B * N * 4
-    d2h = T * d * el + B * d * el
+    e2e = e2e_leg(wl, Kp, M, min(args.steps, 10), flush, world)
 
-    # ---- optional: a stack of decode layers (router GEMM + folded decode layer), stream launches vs one CUDA graph
-    stack = None
-    if args.layers > 0 and world == 1:
-        stack = stack_leg(ex, cfg, layer, tables, (wg, wu, wd), xd, M, args.layers, dev, flush)
-
-    # ---- algorithmic work
-    rows = T * Kp + T * cfg.n_shared
-    flop_layer = rows * 6.0 * d * I
-    flop_gemm1 = rows * 4.0 * d * I
-    pool_bytes = (pool_size + cfg.n_shared) * 3.0 * d * I * el
-    gateup_bytes = pool_bytes * 2.0 / 3.0
     out = {
         "metric": "folded-MoE-layer prefill tokens/s (decode us/layer and roofline fractions alongside)",
         "value": job_tokens_per_s(T, world, pre_ms),
         "unit": "tokens/s",
-        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": pre_ms + dec_ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": cfg.dtype, "data": "synthetic",
@@ -372,72 +695,40 @@ def run_ours(args, rank, world):
                                f"top-{Kp}, prefill T={T}; decode B={B}, pool M={M} (effective {pool_size})",
                    "replicas": world, "l2": "512 MiB buffer read between calls (L2 evicted, lines clean); weights also exceed L2",
                    "logits": cfg.logits, "seed": cfg.seed},
-        "prefill": {"ms": pre_ms, "ms_min": pre_min, "tokens_per_s_per_gpu": T / (pre_ms * 1e-3),
-                    "useful_tflops": flop_layer / (pre_ms * 1e-3) / 1e12,
-                    "frac_of_bf16_peak": flop_layer / (pre_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                    "frac_of_bf16_sustained": flop_layer / (pre_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]},
-        "decode": {"us_per_layer": dec_ms * 1e3, "us_min": dec_min * 1e3, "pool_weight_bytes": pool_bytes,
-                   "layer_gbs": pool_bytes / (dec_ms * 1e-3) / 1e9,
-                   "layer_frac_of_hbm": pool_bytes / (dec_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
-        "kernels_ms": kern,
+        "prefill": pre_rep,
+        "decode": dec_rep,
         "gpu_launches": int(launches),
-        "clocks": sampler.summary(),
-        "e2e": {"value": job_tokens_per_s(T, world, e2e_pre), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
-                "d2h_bytes_per_step": int(d2h), "prefill_ms": e2e_pre, "decode_us": e2e_dec * 1e3},
-        "peaks": {"source": peak_src, **peaks},
-        "wall_s_timed_region": wall,
+        "clocks": clocks,
+        "e2e": e2e,
+        "peaks": {"source": peak_src, **peaks, "nominal": NOMINAL},
+        "wall_s_timed_region": r4(wall),
     }
-    if stack is not None:
-        out["stack"] = stack
-    if "gemm1_gateup_swiglu" in kern:
-        t1 = kern["gemm1_gateup_swiglu"] * 1e-3
-        ach = flop_gemm1 / t1 / 1e12
-        touched = N + cfg.n_shared  # every expert receives rows at these sizes
-        bytes_gemm1 = touched * 2.0 * d * I * el + rows * d * el + rows * I * el
-        out["roofline"] = {"kernel": "grouped GEMM-1 (gate/up + SwiGLU), tcgen05", "bound": "tensor", "achieved": ach,
-                           "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
-                           "traffic": bytes_gemm1 * NCU_TRAFFIC_RATIO["gemm1"],
-                           "traffic_note": "ncu reduced-case DRAM bytes / algorithmic bytes x full-size algorithmic bytes",
-                           "peak_source": f"{peak_src} burst bf16 matmul",
-                           "launch_ms": kern["gemm1_gateup_swiglu"], "flop_per_launch": flop_gemm1}
-    elif "simt_ffn" in kern:
-        t1 = kern["simt_ffn"] * 1e-3
-        ach = flop_layer / t1 / 1e12
-        out["roofline"] = {"kernel": "SIMT fp32 expert FFN", "bound": "alu", "achieved": ach, "peak": 72.0,
-                           "unit": "TFLOP/s", "frac": ach / 72.0, "traffic": None,
-                           "peak_source": "148 SMs x 128 fp32 lanes x 2 x 1.9 GHz"}
-    if "decode_gateup" in kern:
-        tg = kern["decode_gateup"] * 1e-3
-        td = kern.get("decode_down", 0.0) * 1e-3
-        out["decode"]["roofline"] = {"kernel": "decode GEMM-1 (gate/up weight stream over the pool), tcgen05", "bound": "hbm",
-                                     "achieved": gateup_bytes / tg / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                     "frac": gateup_bytes / tg / 1e9 / peaks["hbm_gbs"],
-                                     "traffic": gateup_bytes * NCU_TRAFFIC_RATIO["decode_gateup"],
-                                     "bytes_per_launch": gateup_bytes, "launch_ms": kern["decode_gateup"]}
-        if td > 0:
-            out["decode"]["down_gbs"] = pool_bytes / 3.0 / td / 1e9
-            out["decode"]["ffn_gbs"] = pool_bytes / (tg + td) / 1e9
+    if sustained:
+        out["sustained"] = sustained
+    rl = prefill_roofline(wl, Kp, kern_p, peaks, peak_src, pre_rep["touched_experts"])
+    if rl:
+        out["roofline"] = rl
+    if args.layers > 0 and world == 1:
+        out["stack"] = [stack_leg(wl, M, args.layers, flush), stack_leg(wl, M, args.layers, flush, Kp=Kp)]
 
     # ---- CPU baseline: the oracle as it stands, bounded sample, rank 0 at N=1
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:
-        import oracle
-        per_tok = (Kp + cfg.n_shared) * 6.0 * d * I
-        n_s = int(max(1, min(256, args.cpu_flop_budget / per_tok)))
+        wl.prefill(Kp)
+        wl.decode(M)
+        torch.cuda.synchronize()
+        out["cpu_baseline"], out["parity_sample"] = cpu_baseline_leg(wl, Kp, M, args.cpu_flop_budget)
+
+    # ---- every other benchmark configuration (one GPU, whole-suite run only)
+    if world == 1 and rank == 0 and not args.workload and not args.skip_configs:
+        wl.free()
+        steps_c = min(args.steps, 12)
+        out["configs"] = {}
         t0 = time.time()
-        o = oracle_sample_run(cfg, inp, Kp, M, n_s)
-        yg = y.float().cpu().numpy()[o["idx"]]
-        emax, efro = rel_err(yg, o["y"])
-        out["cpu_baseline"] = {"value": o["tokens_per_s"], "unit": "tokens/s", "cores": oracle.num_threads(),
-                               "kind": "oracle",
-                               "sample": f"{o['tokens']} seeded prefill tokens (all their routes) of the same "
-                                         f"workload; routing at full size; {o['seconds']:.1f}s"}
-        out["parity_sample"] = {"prefill_max_err_rel": emax, "prefill_fro_err_rel": efro, "tokens": int(o["tokens"])}
-        if B * (K + cfg.n_shared) * 6.0 * d * I <= 4 * args.cpu_flop_budget:
-            od = oracle_decode_run(cfg, inp, M)
-            dmax, dfro = rel_err(yd.float().cpu().numpy(), od["y"])
-            out["cpu_baseline"]["decode_us_per_layer"] = od["seconds"] * 1e6
-            out["parity_sample"].update({"decode_max_err_rel": dmax, "decode_fro_err_rel": dfro})
-        log(f"[bench] cpu baseline took {time.time() - t0:.1f}s")
+        for name in ("mixtral", "qwen3", "tiny"):
+            sweep = ((1, 8, 32, 128, 256), (8, 16, 32, 64, 128)) if name == "qwen3" else None
+            out["configs"][name] = measure_config(ex, si.CONFIGS[name], dev, args, peaks, peak_src, flush, steps_c, 3,
+                                                  sweep=sweep, stack_layers=args.layers if name == "qwen3" else 0)
+            log(f"[bench] config {name} done at +{time.time() - t0:.0f}s")
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
@@ -445,54 +736,18 @@ def run_ours(args, rank, world):
 
 
 def run_decode_sweep(args):
-    """Decode batch x pool sweep on one workload's layer (default: the Qwen3-shaped one): us/layer, effective pool,
-    GB/s on the pool's weight bytes, speed-up over the unfolded layer (M = N). One GPU, one JSON line."""
+    """Decode batch x pool sweep on one workload's layer (default: the Qwen3-shaped one). One GPU, one JSON line."""
     import torch
     from paper_2608_24938_b200 import binding as ex
 
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
-    cfg = si.CONFIGS[args.workload]
+    cfg = si.CONFIGS[args.workload or "qwen3"]
     peaks, peak_src = load_peaks()
-    K, N, d, I = cfg.top_k, cfg.n_experts, cfg.hidden, cfg.inter
-    batches = [b for b in (1, 8, 32, 128, 256) if b * K <= 4096]
-    pools = sorted({m for m in (8, 16, 32, 64, 128) if m < N} | {N})
-    inp = build_inputs(cfg, 8, max(batches))
-    g = lambda t: t.to(dev)
-    wg, wu, wd = g(inp["wg"]), g(inp["wu"]), g(inp["wd"])
-    tables = ex.make_tables(*[g(t) for t in inp["tables"]])
-    layer = ex.make_layer(N, cfg.n_shared, d, I, K, cfg.dtype)
-    ws = ex.alloc_workspace(layer, max(batches), K)
-    flush_buf = torch.zeros(128 << 20, dtype=torch.int32, device=dev)
-    el = 2 if cfg.dtype == "bf16" else 4
-    table = []
-    for B in batches:
-        xd, lgd = g(inp["xd"][:B].contiguous()), g(inp["lgd"][:B].contiguous())
-        yd = torch.empty((B, d), dtype=wg.dtype, device=dev)
-        meta = dict(pool_size=torch.zeros(1, dtype=torch.int32, device=dev))
-        row = {}
-        for M in pools:
-            ts = []
-            for it in range(args.steps + max(args.warmup, 3)):
-                torch.sum(flush_buf)
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                ex.exfold_moe_decode(layer, xd, lgd, wg, wu, wd, tables, M, yd, ws, meta=meta)
-                e1.record()
-                torch.cuda.synchronize()
-                if it >= max(args.warmup, 3):
-                    ts.append(e0.elapsed_time(e1))
-            assert ex.exfold_device_status(ws) == 0
-            us = float(np.mean(ts)) * 1e3
-            pool = int(meta["pool_size"].item())
-            byts = (pool + cfg.n_shared) * 3.0 * d * I * el
-            row[M] = {"us": us, "pool": pool, "gbs": byts / (us * 1e-6) / 1e9}
-        for M in pools:
-            r = row[M]
-            table.append({"B": B, "M": M, "effective_pool": r["pool"], "us_per_layer": round(r["us"], 2),
-                          "gbs_on_pool_bytes": round(r["gbs"], 1),
-                          "frac_of_measured_hbm": round(r["gbs"] / peaks["hbm_gbs"], 3),
-                          "speedup_vs_unfolded": round(row[N]["us"] / r["us"], 3)})
+    batches = (1, 8, 32, 128, 256)
+    pools = sorted({m for m in (8, 16, 32, 64, 128) if m < cfg.n_experts} | {cfg.n_experts})
+    wl = Workload(ex, si.scaled(cfg, prefill_tokens=8), dev, batches=batches)
+    table = decode_sweep(wl, batches, pools, peaks, Flush(dev), args.steps, max(args.warmup, 3))
     print(json.dumps({"metric": "decode sweep: us/layer and GB/s on pool weight bytes", "workload": cfg.name,
                       "unit": "us/layer", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
                       "dtype": cfg.dtype, "data": "synthetic", "peaks": {"source": peak_src, **peaks},
@@ -509,13 +764,13 @@ def run_reference(args, rank, world):
     M = args.pool_m or cfg.pool_m[0]
     T, B, K, N, d, I = cfg.prefill_tokens, cfg.decode_batch, cfg.top_k, cfg.n_experts, cfg.hidden, cfg.inter
     inp = build_inputs(cfg, T, B)
-    probe = oracle_sample_run(cfg, inp, Kp, M, max(2, oracle.num_threads()))
+    probe = oracle_sample_run(cfg, inp, Kp, max(2, oracle.num_threads()))
     per_tok = probe["seconds"] / probe["tokens"]
     budget = 150.0 / (args.steps + args.warmup)
     n_s = int(max(1, min(T, 1024, budget / per_tok)))
     times = []
     for it in range(args.warmup + args.steps):
-        r = oracle_sample_run(cfg, inp, Kp, M, n_s, seed=100 + it)
+        r = oracle_sample_run(cfg, inp, Kp, n_s, seed=100 + it)
         if it >= args.warmup:
             times.append(r["seconds"])
     sec = float(np.mean(times))
@@ -538,21 +793,25 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="mixtral", choices=sorted(si.CONFIGS))
+    ap.add_argument("--workload", default=None, choices=sorted(si.CONFIGS),
+                    help="measure only this layer (default: the GLM-4.5-Air-shaped headline plus every other config)")
     ap.add_argument("--k-pre", type=int, default=0)
     ap.add_argument("--pool-m", type=int, default=0)
     ap.add_argument("--tokens", type=int, default=0, help="override the prefill token count (reduced cases for profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the decode batch")
     ap.add_argument("--inter", type=int, default=0, help="override the expert intermediate size")
-    ap.add_argument("--layers", type=int, default=0,
-                    help="also time a stack of this many decode layers (router scores + folded decode layer each), "
-                         "launched on the stream and replayed as one CUDA graph")
+    ap.add_argument("--experts", type=int, default=0, help="override the number of routed experts")
+    ap.add_argument("--layers", type=int, default=4,
+                    help="also time stacks of this many layers (router scores + folded layer each, decode and prefill), "
+                         "launched on the stream and replayed as one CUDA graph (0: skip)")
     ap.add_argument("--decode-sweep", action="store_true",
                     help="instead of the benchmark line: decode batch x pool sweep on --workload (one GPU)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-sustained", action="store_true")
+    ap.add_argument("--skip-configs", action="store_true")
     ap.add_argument("--cpu-flop-budget", type=float, default=3e11,
                     help="flop of oracle work in the cpu-baseline sample (about 10-30 s of CPU time)")
     args = ap.parse_args()

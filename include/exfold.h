@@ -258,6 +258,27 @@ int exfold_router_logits(const exfold_layer *layer, const void *x, const void *w
                          void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * A whole layer from hidden states: the router scores of Eq. 2 (r = W_r x) followed by the folded layer, for
+ * callers that hold the router matrix rather than logits (a stack of layers, each reading the previous
+ * layer's output, captured in one CUDA graph). w_router [N][d] in the layer dtype; `logits` [T][N] fp32 is a
+ * caller-owned device buffer that receives the scores (16-byte aligned; the layer needs them as scratch and
+ * the caller may want them). Everything else as in exfold_moe_prefill / exfold_moe_decode, including the
+ * workspace size. The scores are those of exfold_router_logits, bit for bit: decode batches (and prefill calls of
+ * at most 128 tokens) take the fixed-order dot-product kernel, which joins the decode call's chain of programmatic
+ * dependent launches; longer prefill calls compute the scores with a separate tensor-core launch (a Top-K taken
+ * inside a tensor-core epilogue could not be reproduced bit for bit by another summation order, so the two
+ * steps stay separate kernels there).
+ */
+int exfold_moe_prefill_layer(const exfold_layer *layer, const void *x, const void *w_router, int64_t T,
+                             const void *w_gate, const void *w_up, const void *w_down,
+                             const exfold_tables *tables, int32_t k_pre, float *logits, void *y,
+                             const exfold_prefill_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
+int exfold_moe_decode_layer(const exfold_layer *layer, const void *x, const void *w_router, int64_t B,
+                            const void *w_gate, const void *w_up, const void *w_down,
+                            const exfold_tables *tables, int32_t pool_m, float *logits, void *y,
+                            const exfold_decode_meta *meta, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * The same two calls for activations that live in HOST memory (pinned for real overlap):
  * x_host, logits_host and y_host are host pointers; the call stages them through the
  * workspace with asynchronous copies on the stream (x and logits in before the layer, y out

@@ -31,7 +31,7 @@ EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibr
            "exfold_status_string", "exfold_launch_count", "exfold_profile_enable", "exfold_profile_read",
            "exfold_moe_decode_noalloc", "exfold_static_pool_build", "exfold_moe_decode_static",
            "exfold_moe_prefill_ex", "exfold_router_logits", "exfold_calibrate_layers", "exfold_device_status_noalloc",
-           "exfold_static_scratch_address", "exfold_thread_release"]
+           "exfold_static_scratch_address", "exfold_thread_release", "exfold_moe_prefill_layer", "exfold_moe_decode_layer"]
 PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
                  "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
                  "simt_combine", "gemm1_pair_pass", "gemm2_pair_pass"]
@@ -99,6 +99,12 @@ def _load() -> C.CDLL:
         fn.restype = C.c_int
         fn.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables), i32, vp,
                        C.POINTER(exfold_decode_meta), vp, sz, vp]
+    lib.exfold_moe_prefill_layer.restype = C.c_int
+    lib.exfold_moe_prefill_layer.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables),
+                                             i32, vp, vp, C.POINTER(exfold_prefill_meta), vp, sz, vp]
+    lib.exfold_moe_decode_layer.restype = C.c_int
+    lib.exfold_moe_decode_layer.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables),
+                                            i32, vp, vp, C.POINTER(exfold_decode_meta), vp, sz, vp]
     lib.exfold_moe_decode_noalloc.restype = C.c_int
     lib.exfold_moe_decode_noalloc.argtypes = [C.POINTER(exfold_layer), vp, vp, i64, vp, vp, vp, C.POINTER(exfold_tables),
                                               i32, vp, C.POINTER(exfold_decode_meta), vp]
@@ -288,6 +294,26 @@ def exfold_moe_decode(layer, x, logits, w_gate, w_up, w_down, tables: exfold_tab
                                ws.numel(), _stream(stream))
     if check and rc != 0:
         raise ExfoldError(rc, "exfold_moe_decode")
+    return rc
+
+
+def exfold_moe_prefill_layer(layer, x, w_router, w_gate, w_up, w_down, tables: exfold_tables, k_pre: int, y, ws,
+                             logits_out, meta: Optional[dict] = None, stream=None, check: bool = True) -> int:
+    rc = lib.exfold_moe_prefill_layer(C.byref(layer), _ptr(x), _ptr(w_router), x.shape[0], _ptr(w_gate), _ptr(w_up),
+                                      _ptr(w_down), C.byref(tables), k_pre, _ptr(logits_out), _ptr(y),
+                                      _prefill_meta(meta), _ptr(ws), ws.numel(), _stream(stream))
+    if check and rc != 0:
+        raise ExfoldError(rc, "exfold_moe_prefill_layer")
+    return rc
+
+
+def exfold_moe_decode_layer(layer, x, w_router, w_gate, w_up, w_down, tables: exfold_tables, pool_m: int, y, ws,
+                            logits_out, meta: Optional[dict] = None, stream=None, check: bool = True) -> int:
+    rc = lib.exfold_moe_decode_layer(C.byref(layer), _ptr(x), _ptr(w_router), x.shape[0], _ptr(w_gate), _ptr(w_up),
+                                     _ptr(w_down), C.byref(tables), pool_m, _ptr(logits_out), _ptr(y),
+                                     _decode_meta(meta), _ptr(ws), ws.numel(), _stream(stream))
+    if check and rc != 0:
+        raise ExfoldError(rc, "exfold_moe_decode_layer")
     return rc
 
 

@@ -49,7 +49,7 @@ void prof_reset() {
 
 // ------------------------------------------------------------------ workspace plan
 struct Plan {
-    size_t status, ids, w, omit_src, omit_tgt, block_hist, offsets, work_start, totals, perm, row_tok, row_w,
+    size_t status, ids, w, omit_src, omit_tgt, block_hist, sb_hist, offsets, work_start, totals, perm, row_tok, row_w,
         row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
         xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, calib_warn, total;
 };
@@ -86,6 +86,7 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
     p.omit_src = take((size_t)Tm * l.top_k * 4);
     p.omit_tgt = take((size_t)Tm * l.top_k * 4);
     p.block_hist = take(nblk * N * 4);
+    p.sb_hist = take((nblk + kRouteSuperBlock - 1) / kRouteSuperBlock * N * 4);
     p.offsets = take((G + 2) * 4);
     p.work_start = take((G + 2) * 4);
     p.totals = take(16);
@@ -412,6 +413,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     rp.ids = at<int32_t>(ws, pl.ids); rp.w = at<float>(ws, pl.w);
     rp.omit_src = at<int32_t>(ws, pl.omit_src); rp.omit_tgt = at<int32_t>(ws, pl.omit_tgt);
     rp.block_hist = at<int32_t>(ws, pl.block_hist);
+    rp.sb_hist = at<int32_t>(ws, pl.sb_hist);
     // the first kernel of the call clears the status record (not for the later chunks of a chunked host call)
     rp.status = t_keep_status ? nullptr : at<DeviceStatus>(ws, pl.status);
     { ProfScope ps(0, s); EXFOLD_CUDA(launch_prefill_route(rp, s)); }
@@ -419,7 +421,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     PrefillScatterParams cp{};
     cp.T = T; cp.N = N; cp.n_shared = l.n_shared; cp.Kp = Kp; cp.d_bytes = bf16 ? d * 2 : 0;
     cp.nblk = (int)((T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
-    cp.ids = rp.ids; cp.w = rp.w; cp.block_hist = rp.block_hist;
+    cp.ids = rp.ids; cp.w = rp.w; cp.block_hist = rp.block_hist; cp.sb_hist = rp.sb_hist;
     cp.offsets = at<int32_t>(ws, pl.offsets); cp.work_start = at<int32_t>(ws, pl.work_start);
     cp.x = x; cp.xs = bf16 ? at<char>(ws, pl.xs) : nullptr;
     cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
@@ -670,6 +672,7 @@ static int calibrate_enqueue(const exfold_layer* layer, const void* x_cal, const
         rp.T = m; rp.N = N; rp.K = K; rp.Kp = K; rp.ids = ids; rp.w = at<float>(ws, pl.w);
         rp.loss_thr = INFINITY;
         rp.omit_src = nullptr; rp.omit_tgt = nullptr; rp.block_hist = at<int32_t>(ws, pl.block_hist);
+        rp.sb_hist = at<int32_t>(ws, pl.sb_hist);
         rp.status = nullptr;
         EXFOLD_CUDA(launch_prefill_route(rp, s));
     } else {
@@ -699,6 +702,7 @@ static int calibrate_enqueue(const exfold_layer* layer, const void* x_cal, const
             cp.T = m; cp.N = N; cp.n_shared = 0; cp.Kp = K; cp.d_bytes = d * 2;
             cp.nblk = (int)((m + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
             cp.ids = ids; cp.w = at<float>(ws, pl.w); cp.block_hist = at<int32_t>(ws, pl.block_hist);
+            cp.sb_hist = at<int32_t>(ws, pl.sb_hist);
             cp.offsets = offsets; cp.work_start = work_start;
             cp.x = x_cal; cp.xs = at<char>(ws, pl.xs);
             cp.perm = at<int32_t>(ws, pl.perm); cp.row_tok = at<int32_t>(ws, pl.row_tok);
@@ -799,20 +803,20 @@ int exfold_calibrate_layers(const exfold_layer* layer, const exfold_calib_job* j
     return calibrate_collect(layer, m_max, Ke, n_jobs, unobserved, ws, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
-int exfold_router_logits(const exfold_layer* layer, const void* x, const void* w_router, int64_t T, float* logits,
-                         void* ws, size_t ws_bytes, void* cuda_stream) {
+// Router scores on the stream; `clear_status`: the call stands alone (clears the status record itself)
+static int router_enqueue(const exfold_layer* layer, const void* x, const void* w_router, int64_t T, float* logits,
+                          void* ws, size_t ws_bytes, cudaStream_t s, bool clear_status) {
     if (!valid_layer(layer) || !x || !w_router || !logits || !ws || T < 1) return EXFOLD_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(ws) & 255) != 0 || (reinterpret_cast<uintptr_t>(logits) & 15) != 0)
         return EXFOLD_ERR_INVALID_ARG;
     const exfold_layer& l = *layer;
     const int N = l.n_experts, d = l.hidden;
     if (T > (int64_t)1 << 30) return EXFOLD_ERR_UNSUPPORTED;
-    cudaStream_t s = reinterpret_cast<cudaStream_t>(cuda_stream);
     exfold_layer lc = l;
     lc.n_shared = 0;
     const Plan pl = make_plan(lc, T, 1);
     if (ws_bytes < pl.total) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
-    EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
+    if (clear_status) EXFOLD_CUDA(cudaMemsetAsync(at<char>(ws, pl.status), 0, sizeof(DeviceStatus), s));
     // fp32 layers, and bf16 batches of at most one row tile (decode): dot products in a fixed order. One 128-row
     // tile on the tensor cores would walk the whole K loop on a single SM (10-19 us of latency).
     if (l.dtype == EXFOLD_F32 || (T <= kTileM && aligned16(x) && aligned16(w_router))) {
@@ -837,6 +841,46 @@ int exfold_router_logits(const exfold_layer* layer, const void* x, const void* w
     const int64_t tiles = (T + kTileM - 1) / kTileM;
     EXFOLD_CUDA(launch_grouped_gemm2(g, (int)std::min<int64_t>(sm_count(), tiles), s));
     return EXFOLD_OK;
+}
+
+int exfold_router_logits(const exfold_layer* layer, const void* x, const void* w_router, int64_t T, float* logits,
+                         void* ws, size_t ws_bytes, void* cuda_stream) {
+    return router_enqueue(layer, x, w_router, T, logits, ws, ws_bytes, reinterpret_cast<cudaStream_t>(cuda_stream),
+                          true);
+}
+
+int exfold_moe_prefill_layer(const exfold_layer* layer, const void* x, const void* w_router, int64_t T,
+                             const void* w_gate, const void* w_up, const void* w_down, const exfold_tables* tables,
+                             int32_t k_pre, float* logits, void* y, const exfold_prefill_meta* meta, void* ws,
+                             size_t ws_bytes, void* cuda_stream) {
+    if (!valid_layer(layer) || k_pre < 1 || k_pre > layer->top_k) return EXFOLD_ERR_INVALID_ARG;
+    if (ws_bytes < exfold_workspace_bytes(layer, T < 1 ? 1 : T, k_pre)) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
+    int rc = router_enqueue(layer, x, w_router, T, logits, ws, ws_bytes, reinterpret_cast<cudaStream_t>(cuda_stream),
+                            true);
+    if (rc != EXFOLD_OK) return rc;
+    // the routing kernel would clear the status record again: an error of the router GEMM must stay visible
+    t_keep_status = true;
+    rc = exfold_moe_prefill(layer, x, logits, T, w_gate, w_up, w_down, tables, k_pre, y, meta, ws, ws_bytes, cuda_stream);
+    t_keep_status = false;
+    return rc;
+}
+
+int exfold_moe_decode_layer(const exfold_layer* layer, const void* x, const void* w_router, int64_t B,
+                            const void* w_gate, const void* w_up, const void* w_down, const exfold_tables* tables,
+                            int32_t pool_m, float* logits, void* y, const exfold_decode_meta* meta, void* ws,
+                            size_t ws_bytes, void* cuda_stream) {
+    if (!valid_layer(layer) || !w_router || !logits) return EXFOLD_ERR_INVALID_ARG;
+    if (B < 1 || B > kMaxDecodeBatch) return B < 1 ? EXFOLD_ERR_INVALID_ARG : EXFOLD_ERR_UNSUPPORTED;
+    if (ws_bytes < exfold_workspace_bytes(layer, B, layer->top_k)) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
+    struct PdlScope {
+        PdlScope() { set_pdl(true); }
+        ~PdlScope() { set_pdl(false); }
+    } pdl_scope;  // the router kernel joins the decode call's chain of programmatic dependent launches
+    int rc = router_enqueue(layer, x, w_router, B, logits, ws, ws_bytes, reinterpret_cast<cudaStream_t>(cuda_stream),
+                            false);
+    if (rc != EXFOLD_OK) return rc;
+    return exfold_moe_decode(layer, x, logits, B, w_gate, w_up, w_down, tables, pool_m, y, meta, ws, ws_bytes,
+                             cuda_stream);
 }
 
 int exfold_moe_prefill_host(const exfold_layer* layer, const void* x_host, const float* logits_host, int64_t T,

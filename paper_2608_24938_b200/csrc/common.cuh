@@ -137,10 +137,13 @@ struct PrefillRouteParams {
     int32_t* omit_src;  // [T][K-Kp] or null
     int32_t* omit_tgt;  // [T][K-Kp] or null
     int32_t* block_hist;  // [nblk][N]
+    int32_t* sb_hist;     // [ceil(nblk / kRouteSuperBlock)][N] retained routes per (super-block, expert); the
+                          //   launcher clears it, the blocks add to it
     DeviceStatus* status; // cleared by block 0 (first kernel of a call); may be null
 };
 constexpr int kRouteTokensPerBlock = 32;
 constexpr int kRouteThreads = 512;
+constexpr int kRouteSuperBlock = 64;  // blocks per super-block of the two-level histogram
 
 struct PrefillScatterParams {
     int64_t T;
@@ -149,6 +152,7 @@ struct PrefillScatterParams {
     const int32_t* ids;         // [T][Kp]
     const float* w;             // [T][Kp]
     const int32_t* block_hist;  // [nblk][N] retained routes per (block, expert)
+    const int32_t* sb_hist;     // [ceil(nblk / kRouteSuperBlock)][N] the same per super-block
     int32_t* offsets;           // [G+1] out: first sorted row of each group
     int32_t* work_start;        // [G+1] out: prefix of 128-row tiles per group
     const void* x;      // [T][d]

@@ -137,6 +137,8 @@ __global__ void __launch_bounds__(256) router_simt_kernel(const T* __restrict__ 
                                                           int N, int d, float* __restrict__ out) {
     const int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
+    grid_dep_launch();
+    grid_dep_wait();  // x may be the output of the previous layer's last kernel
     if (w >= Tn * N) return;
     const int64_t i = w / N;
     const int e = (int)(w % N);
@@ -171,13 +173,10 @@ cudaError_t launch_router_simt(const void* x, const void* wr, int dtype, int64_t
     if (warps == 0) return cudaSuccess;
     const unsigned grid = (unsigned)((warps + 7) / 8);
     if (dtype == EXFOLD_BF16)
-        router_simt_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16*>(x),
-                                                reinterpret_cast<const __nv_bfloat16*>(wr), T, N, d, out);
-    else
-        router_simt_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const float*>(x), reinterpret_cast<const float*>(wr), T,
-                                                N, d, out);
-    count_launch();
-    return cudaGetLastError();
+        return launch_pdl(router_simt_kernel<__nv_bfloat16>, grid, 256, 0, s, reinterpret_cast<const __nv_bfloat16*>(x),
+                          reinterpret_cast<const __nv_bfloat16*>(wr), T, N, d, out);
+    return launch_pdl(router_simt_kernel<float>, grid, 256, 0, s, reinterpret_cast<const float*>(x),
+                      reinterpret_cast<const float*>(wr), T, N, d, out);
 }
 
 cudaError_t launch_simt_ffn(const SimtFfnParams& p, cudaStream_t s) {

@@ -4,12 +4,15 @@
 //   route kernel   one warp per token; lane l holds logits l, l+32, ...; after the Top-K
 //                  rounds lane k (k < K) owns route k. Writes ids/w/omitted pairs and a
 //                  per-block histogram of retained experts.
-//   scatter kernel same token->block map as the route kernel. Each block first turns the block
-//                  histograms into its own bases (prefix over experts + prefix over earlier
-//                  blocks; block 0 also publishes offsets and the row-tile prefix for the GEMM
-//                  work list), then ranks its routes in (token, slot) order, so the permutation
-//                  is the stable sort by expert and is bit-reproducible; it also gathers the
-//                  token rows into sorted order.
+//   scatter kernel same token->block map as the route kernel. Each block first derives its own
+//                  bases: the route kernel left one histogram row per block and, added up with
+//                  integer atomics (order-independent), one per super-block of 64 blocks; a block
+//                  sums the super-block rows (all of them: group sizes; those before its own:
+//                  earlier routes) and the at most 63 block rows before it inside its super-block,
+//                  then takes a prefix over experts (block 0 also publishes offsets and the
+//                  row-tile prefix for the GEMM work list). It then ranks its routes in (token,
+//                  slot) order, so the permutation is the stable sort by expert and is
+//                  bit-reproducible; it also gathers the token rows into sorted order.
 #include "common.cuh"
 
 namespace exfold {
@@ -164,44 +167,69 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_route_kernel(PrefillRou
         }
     }
     __syncthreads();
-    for (int e = threadIdx.x; e < N; e += blockDim.x) p.block_hist[(size_t)blockIdx.x * N + e] = hist[e];
+    for (int e = threadIdx.x; e < N; e += blockDim.x) {
+        const int h = hist[e];
+        p.block_hist[(size_t)blockIdx.x * N + e] = h;
+        if (h != 0 && p.sb_hist != nullptr) atomicAdd(&p.sb_hist[(size_t)(blockIdx.x / kRouteSuperBlock) * N + e], h);
+    }
 }
 
 __global__ void __launch_bounds__(kRouteThreads) prefill_scatter_kernel(PrefillScatterParams p) {
     __shared__ int cnt[kMaxExperts];
     __shared__ int pos[kRouteTokensPerBlock * kMaxTopK];
-    __shared__ int part_pre[4][kMaxExperts];  // partial sums over blocks: before this block ...
-    __shared__ int part_tot[4][kMaxExperts];  // ... and over all blocks
-    __shared__ int tot[kMaxExperts];
+    __shared__ int pre[kMaxExperts];  // routes of expert e in earlier blocks
+    __shared__ int tot[kMaxExperts];  // routes of expert e in all blocks
+    __shared__ int warp_tot[kMaxExperts / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int N = p.N, Kp = p.Kp;
     const int64_t tok0 = (int64_t)blockIdx.x * kRouteTokensPerBlock;
     const int ntok = (int)min((int64_t)kRouteTokensPerBlock, p.T - tok0);
     const int n = ntok * Kp;
     const int64_t r0 = tok0 * Kp;
+    for (int e = threadIdx.x; e < N; e += blockDim.x) pre[e] = tot[e] = 0;
+    __syncthreads();
     grid_dep_launch();
     grid_dep_wait();
-    // Every block derives its own bases from the per-block histograms (a few KB, L2-resident): the
-    // first sorted position of expert e for this block is (rows of experts < e) + (rows of e in
-    // earlier blocks). No single-CTA scan kernel sits between routing and the GEMMs.
-    for (int idx = threadIdx.x; idx < 4 * N; idx += blockDim.x) {
-        const int e = idx % N, part = idx / N;
-        int pre = 0, all = 0;
-        for (int b = part; b < p.nblk; b += 4) {
-            const int h = p.block_hist[(size_t)b * N + e];
-            all += h;
-            if (b < (int)blockIdx.x) pre += h;
+    // Bases of this block: first sorted position of expert e = (rows of experts < e) + (rows of e in
+    // earlier blocks). Super-block rows first (nsb of them), then the block rows before this one inside
+    // its super-block: nsb + 63 rows of N counters at most, whatever the token count.
+    {
+        const int sb = (int)blockIdx.x / kRouteSuperBlock, nsb = (p.nblk + kRouteSuperBlock - 1) / kRouteSuperBlock;
+        const int b0 = sb * kRouteSuperBlock, n_inner = (int)blockIdx.x - b0;
+        const int n_rows = nsb + n_inner;
+        for (int idx = threadIdx.x; idx < n_rows * N; idx += blockDim.x) {
+            const int row = idx / N, e = idx - row * N;
+            if (row < nsb) {
+                const int v = p.sb_hist[(size_t)row * N + e];
+                if (v != 0) {
+                    atomicAdd(&tot[e], v);
+                    if (row < sb) atomicAdd(&pre[e], v);
+                }
+            } else {
+                const int v = p.block_hist[(size_t)(b0 + row - nsb) * N + e];
+                if (v != 0) atomicAdd(&pre[e], v);
+            }
         }
-        part_pre[part][e] = pre;
-        part_tot[part][e] = all;
     }
     __syncthreads();
-    for (int e = threadIdx.x; e < N; e += blockDim.x) tot[e] = part_tot[0][e] + part_tot[1][e] + part_tot[2][e] + part_tot[3][e];
+    // exclusive prefix of tot over the experts: warp w scans experts [32w, 32w + 32)
+    if (warp * 32 < N) {
+        const int e = warp * 32 + lane;
+        const int v = e < N ? tot[e] : 0;
+        int incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += u;
+        }
+        if (e < N) cnt[e] = incl - v;
+        if (lane == 31) warp_tot[warp] = incl;
+    }
     __syncthreads();
     for (int e = threadIdx.x; e < N; e += blockDim.x) {
         int off = 0;
-        for (int o = 0; o < e; ++o) off += tot[o];
-        cnt[e] = off + part_pre[0][e] + part_pre[1][e] + part_pre[2][e] + part_pre[3][e];
+        for (int w = 0; w < (e >> 5); ++w) off += warp_tot[w];
+        cnt[e] += off + pre[e];
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {  // group offsets and the row-tile prefix for the GEMM work list
         const int G = N + p.n_shared;
@@ -269,6 +297,11 @@ __global__ void __launch_bounds__(kRouteThreads) prefill_scatter_kernel(PrefillS
 cudaError_t launch_prefill_route(const PrefillRouteParams& p, cudaStream_t s) {
     const int nblk = (int)((p.T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
     const int npl = (p.N + 31) / 32;
+    if (p.sb_hist != nullptr) {  // the super-block histograms are added up with atomics: they start at zero
+        const size_t nsb = (size_t)(nblk + kRouteSuperBlock - 1) / kRouteSuperBlock;
+        cudaError_t e = cudaMemsetAsync(p.sb_hist, 0, nsb * p.N * sizeof(int32_t), s);
+        if (e != cudaSuccess) return e;
+    }
     switch (npl) {
         case 1: return launch_pdl(prefill_route_kernel<1>, nblk, kRouteThreads, 0, s, p);
         case 2: return launch_pdl(prefill_route_kernel<2>, nblk, kRouteThreads, 0, s, p);

@@ -131,7 +131,7 @@ def check_prefill_meta(got, ref):
     """Routing metadata is integer work: bit-exact. Folded weights: fp32 vs double arithmetic."""
     for k in ("ids", "omit_src", "omit_tgt", "perm", "offsets"):
         assert np.array_equal(got[k], ref[k]), f"prefill {k} differs from the oracle"
-    np.testing.assert_allclose(got["w"], ref["w"], rtol=1e-5, atol=1e-5)
+    np.testing.assert_allclose(got["w"], ref["w"], rtol=1e-5, atol=1e-7)
 
 
 def check_decode_meta(got, ref, M):

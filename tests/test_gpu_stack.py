@@ -1,0 +1,204 @@
+"""A stack of folded layers, each fed by the previous one: router scores (Eq. 2: r = W_r x) -> folded layer ->
+next layer's input = this layer's output, every layer with its own expert weights and router matrix. The stack
+runs as plain stream launches and as ONE captured CUDA graph; the oracle runs its own chain (its router scores,
+its folding, its expert outputs, rounded to the layer dtype between layers) from the same first input.
+
+What can be compared: the two chains differ by rounding from the first layer on (bf16 outputs, another summation
+order in the router), so a token's routing is compared where its score gaps exceed the deviation that is observed,
+and outputs are compared on the tokens whose routing has agreed in every layer so far, with the parity tolerance
+growing with depth."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from harness import A, check_output
+
+pytestmark = pytest.mark.gpu
+
+LAYERS = 4
+
+
+def layer_cfg(l, **kw):
+    base = dict(name=f"stack{l}", n_experts=16, n_shared=0, hidden=256, inter=384, top_k=4, dtype="bf16",
+                prefill_tokens=300, k_pre=(2,), decode_batch=24, pool_m=(6,), logits="normal", seed=20260824 + 17 * l)
+    base.update(kw)
+    return si.LayerConfig(**base)
+
+
+class Stack:
+    def __init__(self, n_tokens, **kw):
+        from paper_2608_24938_b200 import binding as ex
+        self.ex, self.dev = ex, torch.device("cuda:0")
+        self.cfgs = [layer_cfg(l, **kw) for l in range(LAYERS)]
+        c0 = self.cfgs[0]
+        self.x0 = si.hidden_states(c0, n_tokens)
+        # expert weights scaled so that a layer roughly keeps the norm of its input
+        self.w = [si.expert_weights(c, std=0.16) for c in self.cfgs]
+        self.wr = [si.router_weights(c, std=4.0 / np.sqrt(c.hidden)) for c in self.cfgs]
+        self.tabs = [si.synthetic_tables(c) for c in self.cfgs]
+        g = lambda t: t.to(self.dev)
+        self.d_w = [tuple(g(t) for t in w) for w in self.w]
+        self.d_wr = [g(t) for t in self.wr]
+        self.d_tabs = [[g(t) for t in tb] for tb in self.tabs]
+        self.tables = [ex.make_tables(*tb) for tb in self.d_tabs]
+        self.layer = ex.make_layer(c0.n_experts, c0.n_shared, c0.hidden, c0.inter, c0.top_k, c0.dtype)
+        self.n = n_tokens
+        self.ws = ex.alloc_workspace(self.layer, n_tokens, c0.top_k)
+        self.ws.fill_(0xFF)
+
+    def buffers(self):
+        c = self.cfgs[0]
+        hs = [self.x0.to(self.dev)] + [torch.full((self.n, c.hidden), float("nan"), dtype=torch.bfloat16,
+                                                  device=self.dev) for _ in range(LAYERS)]
+        lgs = [torch.full((self.n, c.n_experts), float("nan"), device=self.dev) for _ in range(LAYERS)]
+        return hs, lgs
+
+
+def safe_tokens(r64, K, dev_tol):
+    srt = np.sort(r64, axis=1)[:, ::-1]
+    gap = (srt[:, :K] - srt[:, 1:K + 1]).min(axis=1)
+    return gap > 4 * dev_tol
+
+
+def test_decode_stack_stream_graph_and_oracle_chain():
+    st = Stack(24)
+    ex, c = st.ex, st.cfgs[0]
+    B, N, K, M = st.n, c.n_experts, c.top_k, 6
+    i32 = dict(dtype=torch.int32, device=st.dev)
+
+    def run(hs, lgs, metas, stream):
+        for l in range(LAYERS):
+            wg, wu, wd = st.d_w[l]
+            ex.exfold_moe_decode_layer(st.layer, hs[l], st.d_wr[l], wg, wu, wd, st.tables[l], M, hs[l + 1], st.ws,
+                                       logits_out=lgs[l], meta=metas[l], stream=stream)
+
+    def metas_():
+        return [dict(pool_ids=torch.full((M,), -7, **i32), ids=torch.full((B, K), -7, **i32),
+                     w=torch.full((B, K), float("nan"), dtype=torch.float32, device=st.dev)) for _ in range(LAYERS)]
+
+    stream = torch.cuda.Stream()
+    hs_s, lg_s, me_s = *st.buffers(), metas_()
+    hs_g, lg_g, me_g = *st.buffers(), metas_()
+    with torch.cuda.stream(stream):
+        run(hs_s, lg_s, me_s, stream)
+        stream.synchronize()
+        assert ex.exfold_device_status(st.ws, stream) == 0
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            run(hs_g, lg_g, me_g, stream)
+        for _ in range(2):
+            graph.replay()
+        stream.synchronize()
+        assert ex.exfold_device_status(st.ws, stream) == 0
+    # stream launches and graph replay: the first layer sees identical inputs, so everything up to its fp32
+    # accumulator is identical; outputs may differ in the order of the fp32 additions into y (rounding)
+    assert torch.equal(lg_s[0], lg_g[0])
+    for k in ("pool_ids", "ids", "w"):
+        assert torch.equal(me_s[0][k], me_g[0][k]), k
+    for l in range(LAYERS):
+        a, b = hs_s[l + 1].float().cpu().numpy(), hs_g[l + 1].float().cpu().numpy()
+        assert np.isfinite(a).all() and np.isfinite(b).all()
+        assert np.abs(a - b).max() <= 2e-2 * np.abs(a).max()
+
+    # the oracle's own chain
+    x = st.x0
+    agree = np.ones(B, dtype=bool)
+    pools_equal = 0
+    for l in range(LAYERS):
+        cfg = st.cfgs[l]
+        S, L, h, lnh = [t.numpy() for t in st.tabs[l]]
+        wg, wu, wd = st.w[l]
+        r32, r64 = oracle.router_logits(A(x), A(st.wr[l]))
+        ref = oracle.decode_fold(r32, K, M, S, L, h)
+        yref = oracle.moe_apply(A(x), A(wg), A(wu), A(wd), ref["ids"], ref["w"], N, 0)
+        got_lg = lg_s[l].cpu().numpy()
+        dev_tol = np.abs(got_lg - r32)[agree].max() if agree.any() else np.inf
+        if l == 0:
+            assert dev_tol <= 1e-4 * np.abs(r32).max()     # same input: only the summation order differs
+            assert ref["min_gap"] > 1e-6
+        safe = agree & safe_tokens(r64, K, dev_tol)
+        if l == 0:
+            assert safe.all(), "layer 1: the seeded scores have no near-tie, so its whole routing is comparable"
+        same_pool = np.array_equal(me_s[l]["pool_ids"].cpu().numpy(), ref["pool_ids"][:M])
+        if l == 0:
+            assert same_pool
+        if not same_pool:
+            break
+        pools_equal += 1
+        ids = me_s[l]["ids"].cpu().numpy()
+        assert np.array_equal(ids[safe], ref["ids"][safe]), f"layer {l + 1}: remapped ids"
+        np.testing.assert_allclose(me_s[l]["w"].cpu().numpy()[safe], ref["w"][safe], rtol=0.05 * (l + 1), atol=1e-4)
+        y = hs_s[l + 1].float().cpu().numpy()
+        agree = safe & (ids == ref["ids"]).all(axis=1)
+        if agree.any():
+            scale = np.abs(yref).max()
+            assert np.abs(y[agree] - yref[agree]).max() <= 2e-2 * (l + 1) * scale, f"layer {l + 1}: max error"
+            assert np.linalg.norm(y[agree] - yref[agree]) <= 1e-2 * (l + 1) * np.linalg.norm(yref[agree]), \
+                f"layer {l + 1}: Frobenius error"
+        x = torch.from_numpy(yref).to(torch.bfloat16)   # the layer's output dtype
+    assert pools_equal >= 2, "the chains should agree on the pool for the first layers at least"
+
+
+def test_prefill_stack_stream_equals_graph_and_first_layers_match_oracle():
+    st = Stack(300)
+    ex, c = st.ex, st.cfgs[0]
+    T, N, K, Kp = st.n, c.n_experts, c.top_k, 2
+    i32 = dict(dtype=torch.int32, device=st.dev)
+
+    def run(hs, lgs, metas, stream):
+        for l in range(LAYERS):
+            wg, wu, wd = st.d_w[l]
+            ex.exfold_moe_prefill_layer(st.layer, hs[l], st.d_wr[l], wg, wu, wd, st.tables[l], Kp, hs[l + 1], st.ws,
+                                        logits_out=lgs[l], meta=metas[l], stream=stream)
+
+    def metas_():
+        return [dict(ids=torch.full((T, Kp), -7, **i32)) for _ in range(LAYERS)]
+
+    stream = torch.cuda.Stream()
+    hs_s, lg_s, me_s = *st.buffers(), metas_()
+    hs_g, lg_g, me_g = *st.buffers(), metas_()
+    with torch.cuda.stream(stream):
+        run(hs_s, lg_s, me_s, stream)
+        stream.synchronize()
+        assert ex.exfold_device_status(st.ws, stream) == 0
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            run(hs_g, lg_g, me_g, stream)
+        for _ in range(2):
+            graph.replay()
+        stream.synchronize()
+        assert ex.exfold_device_status(st.ws, stream) == 0
+    # the prefill path has no order-dependent arithmetic: stream launches and graph replay agree bit for bit
+    for l in range(LAYERS):
+        assert torch.equal(lg_s[l], lg_g[l]), f"layer {l + 1}: router scores"
+        assert torch.equal(me_s[l]["ids"], me_g[l]["ids"]), f"layer {l + 1}: ids"
+        assert torch.equal(hs_s[l + 1].view(torch.int16), hs_g[l + 1].view(torch.int16)), f"layer {l + 1}: output"
+
+    x = st.x0
+    agree = np.ones(T, dtype=bool)
+    for l in range(LAYERS):
+        S, L, h, lnh = [t.numpy() for t in st.tabs[l]]
+        wg, wu, wd = st.w[l]
+        r32, r64 = oracle.router_logits(A(x), A(st.wr[l]))
+        ref = oracle.prefill_fold(r32, K, Kp, S, L, h, lnh)
+        yref = oracle.moe_apply(A(x), A(wg), A(wu), A(wd), ref["ids"], ref["w"], N, 0)
+        got_lg = lg_s[l].cpu().numpy()
+        dev_tol = np.abs(got_lg - r32)[agree].max()
+        if l == 0:
+            assert dev_tol <= 1e-4 * np.abs(r32).max()
+        # safe against that deviation: the Top-(K+1) score gaps and the gaps between the ranking keys
+        ids_k, _, _ = oracle.gate(r32, K)
+        keys = np.take_along_axis(r64, ids_k.astype(np.int64), 1) + lnh[ids_k]
+        ks = np.sort(keys, axis=1)[:, ::-1]
+        safe = agree & safe_tokens(r64, K, dev_tol) & ((ks[:, :-1] - ks[:, 1:]).min(axis=1) > 4 * dev_tol)
+        ids = me_s[l]["ids"].cpu().numpy()
+        assert np.array_equal(ids[safe], ref["ids"][safe]), f"layer {l + 1}: retained experts"
+        y = hs_s[l + 1].float().cpu().numpy()
+        agree = safe
+        assert agree.mean() > 0.3, f"layer {l + 1}: too few comparable tokens left"
+        scale = np.abs(yref).max()
+        assert np.abs(y[agree] - yref[agree]).max() <= 2e-2 * (l + 1) * scale, f"layer {l + 1}: max error"
+        assert np.linalg.norm(y[agree] - yref[agree]) <= 1e-2 * (l + 1) * np.linalg.norm(yref[agree])
+        x = torch.from_numpy(yref).to(torch.bfloat16)
