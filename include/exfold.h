@@ -367,9 +367,11 @@ int64_t exfold_launch_count(void);
  * (gate/up + SwiGLU), 4 grouped GEMM-2 (down + scatter-combine), 5 fp32->bf16 conversion,
  * 6 decode pool/remap, 7 decode row gather, 8 decode GEMM-1 (gate/up stream), 9 decode GEMM-2 (down stream),
  * 10 SIMT expert FFN, 11 SIMT combine, 12 / 13 the CTA-pair pass of GEMM-1 / GEMM-2 alone (slots 3 and 4 cover a
- * whole GEMM: the pair pass, when it runs, and the one-CTA pass). Returns EXFOLD_OK or EXFOLD_ERR_CUDA.
+ * whole GEMM: the pair pass, when it runs, and the one-CTA pass), 14 decode expert FFN of bf16 layers (one kernel:
+ * pool / remap prologue + gate, up and down weight stream; slot 6 is then the per-token Top-K kernel and slots
+ * 7-9 stay empty). Returns EXFOLD_OK or EXFOLD_ERR_CUDA.
  */
-#define EXFOLD_PROFILE_SLOTS 14
+#define EXFOLD_PROFILE_SLOTS 15
 int exfold_profile_enable(int enable);
 int exfold_profile_read(float *ms, int32_t n_slots);
 

@@ -34,7 +34,7 @@ EXPORTS = ["exfold_workspace_bytes", "exfold_host_staging_bytes", "exfold_calibr
            "exfold_static_scratch_address", "exfold_thread_release", "exfold_moe_prefill_layer", "exfold_moe_decode_layer"]
 PROFILE_SLOTS = ["prefill_route", "prefill_scan", "prefill_scatter", "gemm1_gateup_swiglu", "gemm2_down_combine",
                  "convert_bf16", "decode_route", "decode_gather", "decode_gateup", "decode_down", "simt_ffn",
-                 "simt_combine", "gemm1_pair_pass", "gemm2_pair_pass"]
+                 "simt_combine", "gemm1_pair_pass", "gemm2_pair_pass", "decode_ffn"]
 
 
 class exfold_layer(C.Structure):

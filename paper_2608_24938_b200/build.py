@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libexfold.so")
 SOURCES = ["api.cu", "route_prefill.cu", "route_decode.cu", "ffn_simt.cu", "calibrate.cu", "gemm_prefill.cu",
-           "gemm_pair.cu", "no_alloc.cu"]
+           "gemm_pair.cu", "ffn_decode.cu", "no_alloc.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
 

@@ -51,7 +51,7 @@ void prof_reset() {
 struct Plan {
     size_t status, ids, w, omit_src, omit_tgt, block_hist, sb_hist, offsets, work_start, totals, perm, row_tok, row_w,
         row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
-        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, calib_warn, total;
+        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, calib_warn, w64, total;
 };
 
 bool valid_layer(const exfold_layer* l) {
@@ -95,6 +95,7 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
     p.row_tok = take(Rtot * 4);
     p.row_w = take(Rtot * 4);
     p.row_exp = take(Rtot * 4);
+    p.w64 = take((size_t)std::min<int64_t>(Tm, kMaxDecodeBatch) * l.top_k * 8);  // decode: routed weights in double
     p.pool_ids = take((size_t)N * 4);
     p.pool_size = take(16);
     p.pool_mask = take(32);
@@ -490,7 +491,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
         }
         if (!direct) {
             ProfScope ps(5, s);
-            EXFOLD_CUDA(launch_combine_rows(at<__nv_bfloat16>(ws, pl.obuf), cp.inv_pos, T, Kp, d, l.n_shared,
+            EXFOLD_CUDA(launch_combine_rows(at<__nv_bfloat16>(ws, pl.obuf), cp.inv_pos, T, Kp, d, l.n_shared, nullptr,
                                             reinterpret_cast<__nv_bfloat16*>(y), s));
         }
     } else {
@@ -511,11 +512,15 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     return EXFOLD_OK;
 }
 
+static int router_enqueue(const exfold_layer* layer, const void* x, const void* w_router, int64_t T, float* logits,
+                          void* ws, size_t ws_bytes, cudaStream_t s, bool clear_status);
+
 // Dynamic (tables != null) or static (spool != null) decode step.
+// w_router != null: the router scores are computed first (into `logits`, which is then an output).
 static int decode_impl(const exfold_layer* layer, const void* x, const float* logits, int64_t B, const void* w_gate,
                        const void* w_up, const void* w_down, const exfold_tables* tables,
                        const exfold_static_pool* spool, int32_t pool_m, void* y, const exfold_decode_meta* meta,
-                       void* ws, size_t ws_bytes, void* cuda_stream) {
+                       void* ws, size_t ws_bytes, void* cuda_stream, const void* w_router = nullptr) {
     exfold_tables dummy{};  // the static path needs no tables: satisfy the common pointer checks
     if (spool != nullptr) {
         if (!spool->pool_ids || !spool->target || !spool->scale) return EXFOLD_ERR_INVALID_ARG;
@@ -537,11 +542,10 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
     // a group has at most B rows: the token box of the GEMMs needs only that many (multiple of 32, <= 128)
     const int a_rows = (int)std::min<int64_t>(kTileM, (B + 31) / 32 * 32);
 
-    CUtensorMap tm_xs, tm_wg, tm_wu, tm_h, tm_wd;
+    CUtensorMap tm_wg, tm_wu, tm_h, tm_wd;
     if (bf16) {
         const uint64_t E = (uint64_t)G;
-        bool ok = make_tmap(&tm_xs, at<char>(ws, pl.xs), (uint64_t)max_rows, d, a_rows) &&
-                  make_tmap(&tm_wg, w_gate, E * I, d, 128) && make_tmap(&tm_wu, w_up, E * I, d, 128) &&
+        bool ok = make_tmap(&tm_wg, w_gate, E * I, d, 128) && make_tmap(&tm_wu, w_up, E * I, d, 128) &&
                   make_tmap(&tm_h, at<char>(ws, pl.H), (uint64_t)max_rows, I, a_rows) &&
                   make_tmap(&tm_wd, w_down, E * d, I, 256);
         if (!ok) return EXFOLD_ERR_CUDA;
@@ -565,43 +569,70 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
     rp.grp_expert = at<int32_t>(ws, pl.grp_expert); rp.grp_off = at<int32_t>(ws, pl.grp_off);
     rp.grp_tiles = at<int32_t>(ws, pl.grp_tiles); rp.n_groups = at<int32_t>(ws, pl.n_groups);
     rp.status = at<DeviceStatus>(ws, pl.status);
-    { ProfScope ps(6, s); EXFOLD_CUDA(launch_decode_route(rp, s)); }
-
     if (bf16) {
-        { ProfScope ps(7, s); EXFOLD_CUDA(launch_gather_rows(x, rp.row_tok, rp.n_groups + 1, max_rows, d * 2, at<char>(ws, pl.xs),
-                                       at<float>(ws, pl.y32), (int)B, d, s)); }
-        // The pool's rows (one per distinct (token, pool expert), grouped by pool rank) go through the
-        // same grouped GEMMs as prefill: tokens are the 128-row M operand (mostly padding, which costs
-        // nothing while the kernels are HBM-bound) and every MMA consumes 256 weight rows.
+        // Token-parallel Top-K (with the router scores when w_router is given) -> gate/up kernel that finishes the
+        // routing in its prologue and streams the pool's gate and up weights against x in place -> grouped down
+        // projection over the compact rows -> per-token sum of the rows.
+        int stages = 0, scratch_off = 0, ar = 0;
+        decode_ffn_smem_plan((int)B, K, N, &stages, &scratch_off, &ar);
+        if (stages < 2) return EXFOLD_ERR_UNSUPPORTED;
+        CUtensorMap tm_x, tm_wg64, tm_wu64;
+        const uint64_t E = (uint64_t)G;
+        if (!make_tmap(&tm_x, x, (uint64_t)B, d, ar) || !make_tmap(&tm_wg64, w_gate, E * I, d, 64) ||
+            !make_tmap(&tm_wu64, w_up, E * I, d, 64))
+            return EXFOLD_ERR_CUDA;
+        DecodeTopkParams tp{};
+        tp.logits = logits; tp.x = reinterpret_cast<const __nv_bfloat16*>(x);
+        tp.w_router = reinterpret_cast<const __nv_bfloat16*>(w_router); tp.logits_out = const_cast<float*>(logits);
+        tp.B = (int)B; tp.N = N; tp.K = K; tp.d = d;
+        tp.ids = rp.ids; tp.w64 = at<double>(ws, pl.w64); tp.status = rp.status;
+        { ProfScope ps(6, s); EXFOLD_CUDA(launch_decode_topk(tp, s)); }
+        DecodeFfnParams fp{};
+        fp.tm_x = tm_x; fp.tm_wg = tm_wg; fp.tm_wu = tm_wu; fp.tm_wg64 = tm_wg64; fp.tm_wu64 = tm_wu64;
+        fp.ids = rp.ids; fp.w64 = tp.w64; fp.S = tables->S; fp.L = tables->L; fp.h = tables->h;
+        fp.st_pool = rp.st_pool; fp.st_target = rp.st_target; fp.st_scale = rp.st_scale;
+        fp.B = (int)B; fp.N = N; fp.K = K; fp.M = pool_m; fp.n_shared = l.n_shared; fp.d = d; fp.I = I; fp.a_rows = ar;
+        fp.stages = stages; fp.scratch_off = scratch_off;
+        fp.pool_ids = rp.pool_ids; fp.pool_size = rp.pool_size; fp.pool_mask = rp.pool_mask;
+        // the remapped slots go to a second array: the Top-K ids are read by every CTA while CTA 0 writes
+        fp.out_ids = at<int32_t>(ws, pl.perm); fp.out_w = rp.w; fp.target = rp.target; fp.scale = rp.scale;
+        fp.H = at<__nv_bfloat16>(ws, pl.H); fp.row_tok = rp.row_tok; fp.row_w = rp.row_w;
+        fp.slot_row = at<int32_t>(ws, pl.inv_pos);
+        fp.grp_expert = rp.grp_expert; fp.grp_off = rp.grp_off; fp.grp_tiles = rp.grp_tiles; fp.n_groups = rp.n_groups;
+        fp.status = rp.status;
+        { ProfScope ps(14, s); EXFOLD_CUDA(launch_decode_ffn(fp, sm_count(), s)); }
+        // Down projection on the grouped GEMM-2 kernel over the compact rows (the whole intermediate dimension is
+        // its K, so no partial outputs meet in memory); each row's weighted output is stored once, in bf16, and a
+        // token's rows are then summed in slot order: no atomics, so a decode step is reproducible bit for bit.
         const int max_groups = std::min(pool_m, N) + l.n_shared;
         const int tiles_per_group = (int)((B + kTileM - 1) / kTileM);
         const int sms = std::min(sm_count(), kMaxCtas);
         GroupedGemmParams g{};
-        g.tm_a = tm_xs; g.tm_a2 = tm_xs; g.tm_b0 = tm_wg; g.tm_b1 = tm_wu; g.x_rows = 1; g.o32 = nullptr;
+        g.tm_a = tm_h; g.tm_a2 = tm_h; g.tm_b0 = tm_wd; g.tm_b1 = tm_wd; g.x_rows = 1; g.o32 = nullptr;
         g.offsets = rp.grp_off; g.work_start = rp.grp_tiles; g.G = max_groups; g.n_routed = 0x7fffffff;
-        g.R = max_rows; g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.a_rows = a_rows;
+        g.R = max_rows; g.d = d; g.I = I; g.n_ntiles = (d + 255) / 256; g.ksplit = 1; g.a_rows = a_rows;
         g.grp_expert = rp.grp_expert; g.n_groups_dev = rp.n_groups;
-        g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = rp.row_tok; g.row_w = rp.row_w;
-        g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
-        const int64_t items1 = (int64_t)max_groups * tiles_per_group * g.n_ntiles;
-        { ProfScope ps(8, s); EXFOLD_CUDA(launch_grouped_gemm1(g, (int)std::min<int64_t>(sms, items1), s)); }
-        g.tm_a = tm_h; g.tm_b0 = tm_wd; g.n_ntiles = (d + 255) / 256;
-        g.y32 = at<float>(ws, pl.y32); g.y = reinterpret_cast<__nv_bfloat16*>(y); g.store_rows = 0;
-        // split K so that every SM streams a share of W_down even with few (expert, column tile) items
-        const int nkb2 = I / 64;
-        const int64_t base_items = (int64_t)max_groups * tiles_per_group * g.n_ntiles;
-        int ks = (int)((2 * (int64_t)sms + base_items - 1) / base_items);
-        ks = std::max(1, std::min(ks, nkb2 / 4));
-        const int kb_per = (nkb2 + ks - 1) / ks;
-        g.ksplit = (nkb2 + kb_per - 1) / kb_per;  // no empty parts
-        { ProfScope ps(9, s); EXFOLD_CUDA(launch_grouped_gemm2(g, (int)std::min<int64_t>(sms, base_items * g.ksplit), s)); }
-        { ProfScope ps(5, s); EXFOLD_CUDA(launch_convert_bf16(at<float>(ws, pl.y32), B * d, y, s)); }
+        g.H = fp.H; g.row_tok = rp.row_tok; g.row_w = rp.row_w;
+        g.y32 = nullptr; g.y = at<__nv_bfloat16>(ws, pl.obuf); g.store_rows = 1; g.status = rp.status;
+        const int64_t items2 = (int64_t)max_groups * tiles_per_group * g.n_ntiles;
+        { ProfScope ps(9, s); EXFOLD_CUDA(launch_grouped_gemm2(g, (int)std::min<int64_t>(sms, items2), s)); }
+        { ProfScope ps(5, s); EXFOLD_CUDA(launch_combine_rows(g.y, fp.slot_row, B, K, d, l.n_shared, rp.n_groups + 2,
+                                                       reinterpret_cast<__nv_bfloat16*>(y), s)); }
+        rp.ids = fp.out_ids;  // for the metadata copies below
     } else {
+    if (w_router != nullptr) {
+        rc = router_enqueue(layer, x, w_router, B, const_cast<float*>(logits), ws, ws_bytes, s, false);
+        if (rc != EXFOLD_OK) return rc;
+    }
+    { ProfScope ps(6, s); EXFOLD_CUDA(launch_decode_route(rp, s)); }
+
+    {
         SimtFfnParams fp{};
         fp.x = x; fp.wg = w_gate; fp.wu = w_up; fp.wd = w_down; fp.dtype = l.dtype; fp.d = d; fp.I = I;
         fp.T = B; fp.Kr = K; fp.n_shared = l.n_shared; fp.N = N; fp.ids = rp.ids; fp.out = at<float>(ws, pl.out);
         { ProfScope ps(10, s); EXFOLD_CUDA(launch_simt_ffn(fp, s)); }
         { ProfScope ps(11, s); EXFOLD_CUDA(launch_combine_routes(fp.out, rp.w, B, K, d, l.n_shared, y, l.dtype, s)); }
+    }
     }
     if (meta) {
         if ((rc = copy_meta(meta->pool_ids, rp.pool_ids, (size_t)pool_m * 4, s))) return rc;
@@ -872,15 +903,9 @@ int exfold_moe_decode_layer(const exfold_layer* layer, const void* x, const void
     if (!valid_layer(layer) || !w_router || !logits) return EXFOLD_ERR_INVALID_ARG;
     if (B < 1 || B > kMaxDecodeBatch) return B < 1 ? EXFOLD_ERR_INVALID_ARG : EXFOLD_ERR_UNSUPPORTED;
     if (ws_bytes < exfold_workspace_bytes(layer, B, layer->top_k)) return EXFOLD_ERR_WORKSPACE_TOO_SMALL;
-    struct PdlScope {
-        PdlScope() { set_pdl(true); }
-        ~PdlScope() { set_pdl(false); }
-    } pdl_scope;  // the router kernel joins the decode call's chain of programmatic dependent launches
-    int rc = router_enqueue(layer, x, w_router, B, logits, ws, ws_bytes, reinterpret_cast<cudaStream_t>(cuda_stream),
-                            false);
-    if (rc != EXFOLD_OK) return rc;
-    return exfold_moe_decode(layer, x, logits, B, w_gate, w_up, w_down, tables, pool_m, y, meta, ws, ws_bytes,
-                             cuda_stream);
+    if ((reinterpret_cast<uintptr_t>(logits) & 15) != 0 || !aligned16(w_router)) return EXFOLD_ERR_INVALID_ARG;
+    return decode_impl(layer, x, logits, B, w_gate, w_up, w_down, tables, nullptr, pool_m, y, meta, ws, ws_bytes,
+                       cuda_stream, w_router);
 }
 
 int exfold_moe_prefill_host(const exfold_layer* layer, const void* x_host, const float* logits_host, int64_t T,

@@ -58,8 +58,10 @@ bool pdl_enabled();
 
 // Order-preserving map float -> uint32 (larger float <=> larger key), so warp arg-max / arg-min can use
 // the hardware integer reductions (redux.sync) instead of shuffle trees.
+// -0.0 and +0.0 compare equal as floats, so they get one key (a tie, which the lower expert id then wins).
 __device__ __forceinline__ uint32_t float_order_key(float f) {
-    const uint32_t b = __float_as_uint(f);
+    uint32_t b = __float_as_uint(f);
+    if (b == 0x80000000u) b = 0u;
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 __device__ __forceinline__ float float_from_order_key(uint32_t k) {
@@ -196,11 +198,64 @@ struct DecodeRouteParams {
     DeviceStatus* status; // cleared here (first kernel of a decode call)
 };
 cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s);
+
+// Token-parallel half of decode routing for bf16 layers (one CTA per token): optional router scores, Top-K,
+// softmax weights in double; clears the status record
+struct DecodeTopkParams {
+    const float* logits;            // [B][N] (w_router == null)
+    const __nv_bfloat16* x;         // [B][d]  (w_router != null)
+    const __nv_bfloat16* w_router;  // [N][d] or null
+    float* logits_out;              // [B][N] (w_router != null)
+    int B, N, K, d;
+    int32_t* ids;   // [B][K] routed experts in router order
+    double* w64;    // [B][K] their softmax weights
+    DeviceStatus* status;
+};
+cudaError_t launch_decode_topk(const DecodeTopkParams& p, cudaStream_t s);
+
+// Decode, bf16 layers: the gate/up half of the expert FFN over the pool. The kernel finishes the routing in its
+// prologue (every CTA: pool of Eq. 11 from the routed weights, minimum-loss targets of Eq. 12, remap of Eq. 14,
+// rows per group), streams the pool's gate and up weights once against x read in place, and leaves H (compact rows)
+// and the execution lists for the grouped down projection (ffn_decode.cu)
+struct DecodeFfnParams {
+    CUtensorMap tm_x;     // x [B][d], box a_rows x 64
+    CUtensorMap tm_wg;    // W_gate as [(E*I)][d], box 128 x 64
+    CUtensorMap tm_wu;    // W_up
+    CUtensorMap tm_wg64;  // the same with 64-row boxes (half-width items)
+    CUtensorMap tm_wu64;
+    const int32_t* ids;   // [B][K] from the top-k kernel
+    const double* w64;    // [B][K]
+    const float* S;       // tables (dynamic pool)
+    const float* L;
+    const float* h;
+    const int32_t* st_pool;    // static pool (all null for the dynamic pool)
+    const int32_t* st_target;
+    const float* st_scale;
+    int B, N, K, M, n_shared, d, I, a_rows;
+    int stages, scratch_off;  // shared-memory plan made by the launcher
+    // metadata written by CTA 0 (workspace copies)
+    int32_t* pool_ids;    // [N] (-1 padded)
+    int32_t* pool_size;   // [1]
+    uint32_t* pool_mask;  // [8]
+    int32_t* out_ids;     // [B][K] remapped
+    float* out_w;         // [B][K]
+    int32_t* target;      // [N]
+    float* scale;         // [N]
+    // execution lists: one row per distinct (token, pool expert), grouped by pool rank (shared expert last)
+    __nv_bfloat16* H;     // [rows][I]
+    int32_t* row_tok;     // [rows]
+    float* row_w;         // [rows] merged weight of the row
+    int32_t* slot_row;    // [B][K] row of each routed slot, -1 for a slot merged into an earlier one
+    int32_t* grp_expert;  // [G]
+    int32_t* grp_off;     // [G+1]
+    int32_t* grp_tiles;   // [G+1] prefix of 128-row tiles per group
+    int32_t* n_groups;    // [3]: groups, rows, first row of the shared expert's group
+    DeviceStatus* status;
+};
+cudaError_t launch_decode_ffn(const DecodeFfnParams& p, int sms, cudaStream_t s);
+size_t decode_ffn_smem_plan(int B, int K, int N, int* stages, int* scratch_off, int* a_rows);
 cudaError_t launch_static_pool(int N, int M, const float* S, const float* L, const float* h, int32_t* pool_ids,
                                int32_t* target, float* scale, cudaStream_t s);
-cudaError_t launch_gather_rows(const void* x, const int32_t* row_tok, const int32_t* n_rows_ptr, int max_rows,
-                               int row_bytes, void* xs, float* y32, int zero_rows, int zero_row_floats,
-                               cudaStream_t s);
 
 // ---------------------------------------------------------------- SIMT expert FFN (fp32 accumulate)
 struct SimtFfnParams {
@@ -221,10 +276,10 @@ cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, i
                                   void* y, int dtype, cudaStream_t s);
 cudaError_t launch_router_simt(const void* x, const void* wr, int dtype, int64_t T, int N, int d, float* out,
                                cudaStream_t s);
-cudaError_t launch_convert_bf16(const float* y32, int64_t n, void* y, cudaStream_t s);
-// y[i] = sum_j O[inv_pos[i*Kr+j]] (+ O[R+i] for the shared expert), fp32 sum in slot order, bf16 out
+// y[i] = sum_j O[inv_pos[i*Kr+j]] (entries < 0 skipped) (+ O[shared0 + i] for the shared expert), fp32 sum in slot
+// order, bf16 out. shared0 = T*Kr, or *shared0_dev when that is given (decode: known only on the device).
 cudaError_t launch_combine_rows(const __nv_bfloat16* O, const int32_t* inv_pos, int64_t T, int Kr, int d,
-                                int n_shared, __nv_bfloat16* y, cudaStream_t s);
+                                int n_shared, const int32_t* shared0_dev, __nv_bfloat16* y, cudaStream_t s);
 
 // ---------------------------------------------------------------- calibration
 struct CalibStatsParams {

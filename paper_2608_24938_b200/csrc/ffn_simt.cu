@@ -88,15 +88,18 @@ __global__ void combine_routes_kernel(const float* __restrict__ out, const float
 // expert; a token's routes are found through the inverse permutation and summed in fp32, slot order.
 __global__ void __launch_bounds__(256) combine_rows_kernel(const __nv_bfloat16* __restrict__ O,
                                                            const int32_t* __restrict__ inv_pos, int64_t Tn, int Kr, int d,
-                                                           int n_shared, __nv_bfloat16* __restrict__ y) {
+                                                           int n_shared, const int32_t* __restrict__ shared0_dev,
+                                                           __nv_bfloat16* __restrict__ y) {
     const int64_t i = blockIdx.x;
     grid_dep_launch();
     grid_dep_wait();
+    const int64_t shared0 = shared0_dev != nullptr ? (int64_t)*shared0_dev : Tn * Kr;
     for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int j = 0; j <= Kr; ++j) {
             if (j == Kr && !n_shared) break;
-            const int64_t row = j < Kr ? (int64_t)inv_pos[i * Kr + j] : Tn * Kr + i;
+            const int64_t row = j < Kr ? (int64_t)inv_pos[i * Kr + j] : shared0 + i;
+            if (row < 0) continue;  // a slot merged into an earlier one of the same token
             const uint4 v = *reinterpret_cast<const uint4*>(O + row * d + c);
             const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v);
 #pragma unroll
@@ -111,22 +114,6 @@ __global__ void __launch_bounds__(256) combine_rows_kernel(const __nv_bfloat16* 
 #pragma unroll
         for (int u = 0; u < 4; ++u) o2[u] = __floats2bfloat162_rn(acc[2 * u], acc[2 * u + 1]);
         *reinterpret_cast<uint4*>(y + i * d + c) = o;
-    }
-}
-
-__global__ void convert_bf16_kernel(const float4* __restrict__ src, int64_t n4, uint2* __restrict__ dst) {
-    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    grid_dep_launch();
-    grid_dep_wait();
-    for (; i < n4; i += stride) {
-        float4 v = src[i];
-        __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y);
-        __nv_bfloat162 b = __floats2bfloat162_rn(v.z, v.w);
-        uint2 o;
-        o.x = *reinterpret_cast<uint32_t*>(&a);
-        o.y = *reinterpret_cast<uint32_t*>(&b);
-        dst[i] = o;
     }
 }
 
@@ -207,18 +194,9 @@ cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, i
 }
 
 cudaError_t launch_combine_rows(const __nv_bfloat16* O, const int32_t* inv_pos, int64_t T, int Kr, int d,
-                                int n_shared, __nv_bfloat16* y, cudaStream_t s) {
+                                int n_shared, const int32_t* shared0_dev, __nv_bfloat16* y, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
-    return launch_pdl(combine_rows_kernel, (unsigned)T, 256, 0, s, O, inv_pos, T, Kr, d, n_shared, y);
-}
-
-cudaError_t launch_convert_bf16(const float* y32, int64_t n, void* y, cudaStream_t s) {
-    if (n == 0) return cudaSuccess;
-    const int64_t n4 = n / 4;  // n is a multiple of 64 (d is)
-    int blocks = (int)((n4 + 255) / 256);
-    if (blocks > 148 * 16) blocks = 148 * 16;
-    return launch_pdl(convert_bf16_kernel, blocks, 256, 0, s, reinterpret_cast<const float4*>(y32), n4,
-                      reinterpret_cast<uint2*>(y));
+    return launch_pdl(combine_rows_kernel, (unsigned)T, 256, 0, s, O, inv_pos, T, Kr, d, n_shared, shared0_dev, y);
 }
 
 }  // namespace exfold

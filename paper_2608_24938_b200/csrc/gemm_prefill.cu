@@ -451,7 +451,7 @@ static cudaError_t launch_gemm_t(const GroupedGemmParams& p, int grid, cudaStrea
 }
 
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s) {
-    return p.grp_expert != nullptr ? launch_gemm_t<0, true>(p, grid, s) : launch_gemm_t<0, false>(p, grid, s);
+    return launch_gemm_t<0, false>(p, grid, s);  // decode has its own gate/up kernel (ffn_decode.cu)
 }
 cudaError_t launch_grouped_gemm2(const GroupedGemmParams& p, int grid, cudaStream_t s) {
     return p.grp_expert != nullptr ? launch_gemm_t<1, true>(p, grid, s) : launch_gemm_t<1, false>(p, grid, s);

@@ -338,6 +338,90 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
 }
 
 
+// ---------------------------------------------------------------- token-parallel first half of decode routing
+// One CTA per token: (optionally) the router scores of Eq. 2 as fixed-order dot products - the same lane
+// partition, the same fused multiply-adds and the same shuffle tree as router_simt_kernel, so the scores are
+// those of exfold_router_logits bit for bit -, then the token's Top-K and its softmax weights in double
+// (slot order). CTA 0 also clears the status record.
+// The batch-level half (pool, targets, remap) runs in the prologue of the expert-FFN kernel (ffn_decode.cu).
+template <int NPL>
+__global__ void __launch_bounds__(256) decode_topk_kernel(DecodeTopkParams p) {
+    __shared__ float s_lg[kMaxExperts];
+    const int i = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int N = p.N, K = p.K, d = p.d;
+    grid_dep_launch();
+    grid_dep_wait();  // x may be the previous layer's output; the workspace may still be read by the previous call
+    if (i == 0 && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
+    if (p.w_router != nullptr) {
+        const __nv_bfloat16* xi = p.x + (size_t)i * d;
+        for (int e = warp; e < N; e += 8) {
+            const __nv_bfloat16* we = p.w_router + (size_t)e * d;
+            float acc = 0.f;
+            for (int c = lane * 8; c < d; c += 256) {
+                const uint4 a = *reinterpret_cast<const uint4*>(we + c), b = *reinterpret_cast<const uint4*>(xi + c);
+                const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+                const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float2 fa = __bfloat1622float2(pa[j]), fb = __bfloat1622float2(pb[j]);
+                    acc = fmaf(fa.x, fb.x, acc);
+                    acc = fmaf(fa.y, fb.y, acc);
+                }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            if (lane == 0) {
+                s_lg[e] = acc;
+                p.logits_out[(size_t)i * N + e] = acc;
+            }
+        }
+        __syncthreads();
+    }
+    if (warp != 0) return;
+    float v[NPL];
+#pragma unroll
+    for (int q = 0; q < NPL; ++q) {
+        const int e = lane + 32 * q;
+        v[q] = e < N ? (p.w_router != nullptr ? s_lg[e] : p.logits[(size_t)i * N + e]) : -INFINITY;
+    }
+    uint32_t key_q[NPL];
+    uint32_t used = 0;
+#pragma unroll
+    for (int q = 0; q < NPL; ++q) {
+        key_q[q] = float_order_key(v[q]);
+        if (lane + 32 * q >= N) used |= 1u << q;
+    }
+    int my_id = -1;
+    float my_r = 0.f;
+    for (int k = 0; k < K; ++k) {
+        uint32_t bk = 0;
+        int be = 0x7fffffff;
+#pragma unroll
+        for (int q = 0; q < NPL; ++q) {
+            const bool free_q = !((used >> q) & 1u);
+            if (free_q && (be == 0x7fffffff || key_q[q] > bk)) {
+                bk = key_q[q];
+                be = lane + 32 * q;
+            }
+        }
+        uint32_t mk;
+        be = warp_argmax(be != 0x7fffffff, bk, be, &mk);
+        if ((be & 31) == lane) used |= 1u << (be >> 5);
+        if (lane == k) {
+            my_id = be;
+            my_r = float_from_order_key(mk);
+        }
+    }
+    const float rmax = __shfl_sync(0xffffffffu, my_r, 0);
+    const double ex = lane < K ? exp((double)my_r - (double)rmax) : 0.0;
+    double sum = 0.0;
+    for (int k = 0; k < K; ++k) sum += __shfl_sync(0xffffffffu, ex, k);  // slot order, like the definition
+    if (lane < K) {
+        p.ids[(size_t)i * K + lane] = my_id;
+        p.w64[(size_t)i * K + lane] = ex / sum;
+    }
+}
+
 // Static pool: pool = TopK_e(h_e, M) (ties -> lower id, descending h), then Eq. 12 for every source.
 __global__ void __launch_bounds__(256) static_pool_kernel(int N, int M, const float* __restrict__ S,
                                                           const float* __restrict__ L, const float* __restrict__ h,
@@ -387,27 +471,6 @@ __global__ void __launch_bounds__(256) static_pool_kernel(int N, int M, const fl
     }
 }
 
-// xs[row] = x[row_tok[row]] for row < n_rows (device value); CTAs with blockIdx < zero_rows also
-// clear one row of the fp32 accumulator y32.
-__global__ void __launch_bounds__(256) gather_rows_kernel(const void* __restrict__ x,
-                                                          const int32_t* __restrict__ row_tok,
-                                                          const int32_t* __restrict__ n_rows_ptr, int row_bytes,
-                                                          void* __restrict__ xs, float* __restrict__ y32,
-                                                          int zero_rows, int zero_row_floats) {
-    const int row = blockIdx.x;
-    grid_dep_launch();
-    grid_dep_wait();
-    if (y32 != nullptr && row < zero_rows) {
-        float4* z = reinterpret_cast<float4*>(y32 + (size_t)row * zero_row_floats);
-        for (int c = threadIdx.x; c < zero_row_floats / 4; c += blockDim.x) z[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    if (row >= *n_rows_ptr) return;
-    const uint4* src =
-        reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(x) + (size_t)row_tok[row] * row_bytes);
-    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<char*>(xs) + (size_t)row * row_bytes);
-    for (int c = threadIdx.x; c < (row_bytes >> 4); c += blockDim.x) dst[c] = __ldg(src + c);
-}
-
 }  // namespace
 
 cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s) {
@@ -430,18 +493,19 @@ cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s) {
     return err;
 }
 
+cudaError_t launch_decode_topk(const DecodeTopkParams& p, cudaStream_t s) {
+    const int npl = (p.N + 31) / 32;
+    switch (npl) {
+        case 1: return launch_pdl(decode_topk_kernel<1>, p.B, 256, 0, s, p);
+        case 2: return launch_pdl(decode_topk_kernel<2>, p.B, 256, 0, s, p);
+        case 3: case 4: return launch_pdl(decode_topk_kernel<4>, p.B, 256, 0, s, p);
+        default: return launch_pdl(decode_topk_kernel<8>, p.B, 256, 0, s, p);
+    }
+}
+
 cudaError_t launch_static_pool(int N, int M, const float* S, const float* L, const float* h, int32_t* pool_ids,
                                int32_t* target, float* scale, cudaStream_t s) {
     return launch_pdl(static_pool_kernel, 1, 256, 0, s, N, M, S, L, h, pool_ids, target, scale);
-}
-
-cudaError_t launch_gather_rows(const void* x, const int32_t* row_tok, const int32_t* n_rows_ptr, int max_rows,
-                               int row_bytes, void* xs, float* y32, int zero_rows, int zero_row_floats,
-                               cudaStream_t s) {
-    int grid = max_rows > zero_rows ? max_rows : zero_rows;
-    if (grid == 0) return cudaSuccess;
-    return launch_pdl(gather_rows_kernel, grid, 256, 0, s, x, row_tok, n_rows_ptr, row_bytes, xs, y32, zero_rows,
-                      zero_row_floats);
 }
 
 }  // namespace exfold
