@@ -491,7 +491,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
         }
         if (!direct) {
             ProfScope ps(5, s);
-            EXFOLD_CUDA(launch_combine_rows(at<__nv_bfloat16>(ws, pl.obuf), cp.inv_pos, T, Kp, d, l.n_shared, nullptr,
+            EXFOLD_CUDA(launch_combine_rows(at<__nv_bfloat16>(ws, pl.obuf), cp.inv_pos, T, Kp, d, l.n_shared, nullptr, 1, 0,
                                             reinterpret_cast<__nv_bfloat16*>(y), s));
         }
     } else {
@@ -614,10 +614,16 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
         g.grp_expert = rp.grp_expert; g.n_groups_dev = rp.n_groups;
         g.H = fp.H; g.row_tok = rp.row_tok; g.row_w = rp.row_w;
         g.y32 = nullptr; g.y = at<__nv_bfloat16>(ws, pl.obuf); g.store_rows = 1; g.status = rp.status;
-        const int64_t items2 = (int64_t)max_groups * tiles_per_group * g.n_ntiles;
-        { ProfScope ps(9, s); EXFOLD_CUDA(launch_grouped_gemm2(g, (int)std::min<int64_t>(sms, items2), s)); }
-        { ProfScope ps(5, s); EXFOLD_CUDA(launch_combine_rows(g.y, fp.slot_row, B, K, d, l.n_shared, rp.n_groups + 2,
-                                                       reinterpret_cast<__nv_bfloat16*>(y), s)); }
+        // Fewer (expert, column tile) items than half the SMs (few experts, large I): K is split in two so that
+        // enough SMs stream W_down; each part's rows go to a plane of their own (the two planes are the row buffer
+        // and the unused gathered-rows region before it) and are summed, in order, by the kernel after.
+        const int nkb2 = I / 64;
+        const int64_t base_items = (int64_t)max_groups * tiles_per_group * g.n_ntiles;
+        g.ksplit = (2 * base_items < sms && nkb2 >= 8) ? kMaxDecodeKsplit : 1;
+        g.y = g.ksplit > 1 ? at<__nv_bfloat16>(ws, pl.obuf) - (size_t)max_rows * d : at<__nv_bfloat16>(ws, pl.obuf);
+        { ProfScope ps(9, s); EXFOLD_CUDA(launch_grouped_gemm2(g, (int)std::min<int64_t>(sms, base_items * g.ksplit), s)); }
+        { ProfScope ps(5, s); EXFOLD_CUDA(launch_combine_rows(g.y, fp.slot_row, B, K, d, l.n_shared, rp.n_groups + 2, g.ksplit,
+                                                       max_rows, reinterpret_cast<__nv_bfloat16*>(y), s)); }
         rp.ids = fp.out_ids;  // for the metadata copies below
     } else {
     if (w_router != nullptr) {

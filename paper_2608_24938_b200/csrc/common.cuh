@@ -277,9 +277,12 @@ cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, i
 cudaError_t launch_router_simt(const void* x, const void* wr, int dtype, int64_t T, int N, int d, float* out,
                                cudaStream_t s);
 // y[i] = sum_j O[inv_pos[i*Kr+j]] (entries < 0 skipped) (+ O[shared0 + i] for the shared expert), fp32 sum in slot
-// order, bf16 out. shared0 = T*Kr, or *shared0_dev when that is given (decode: known only on the device).
+// order, bf16 out. shared0 = T*Kr, or *shared0_dev when that is given (decode: known only on the device). A row may
+// be stored as `parts` partial rows (decode's K split), part k at row k * part_rows + row: summed in that order.
 cudaError_t launch_combine_rows(const __nv_bfloat16* O, const int32_t* inv_pos, int64_t T, int Kr, int d,
-                                int n_shared, const int32_t* shared0_dev, __nv_bfloat16* y, cudaStream_t s);
+                                int n_shared, const int32_t* shared0_dev, int parts, int64_t part_rows,
+                                __nv_bfloat16* y, cudaStream_t s);
+constexpr int kMaxDecodeKsplit = 2;
 
 // ---------------------------------------------------------------- calibration
 struct CalibStatsParams {

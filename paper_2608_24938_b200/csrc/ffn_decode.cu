@@ -70,20 +70,40 @@ struct Item {
 struct Sched {  // the same in every role of a CTA
     int n_pairs, nfull, has_half, f_keep, split, total;
     int identity;  // pair p is (group p, token tile 0): no list needed
+    int ctas;      // CTAs that take work: item w belongs to CTA w % ctas
 };
 
+// Two ways to deal F full items (plus a few natural halves) over the grid, both static:
+//   (a) all CTAs, the last partial round of r full items cut into 2r halves when every half finds its own SM;
+//   (b) only eff = ceil(F / rounds) CTAs, each exactly `rounds` items, so that all of them finish together.
+// In units of the time one SM needs for a full item alone, a phase of n SMs working at once takes z * max(1, n / c)
+// for items of size z: about c = 110 streaming SMs saturate HBM (measured: ~55 GB/s per SM, ~6 TB/s together).
+// (b) wins when the remainder would leave a few SMs working alone (448 items: 112 x 4 rather than 148 x 3 + 8 halves).
 __device__ __forceinline__ Sched make_sched(int n_pairs, int I, int grid, int identity) {
     Sched sc;
     sc.identity = identity;
     sc.n_pairs = n_pairs;
     sc.nfull = I / 128;
     sc.has_half = (I % 128) != 0 ? 1 : 0;
-    const int F = n_pairs * sc.nfull;
-    const int r = F % grid;
-    // the last partial round of full items, as halves, if every half then finds an SM of its own
-    sc.split = (r > 0 && 2 * r + n_pairs * sc.has_half <= grid) ? r : 0;
+    const int F = n_pairs * sc.nfull, H = n_pairs * sc.has_half;
+    const float c = 110.0f;
+    const int q = F / grid, r = F % grid;
+    const bool can_split = r > 0 && 2 * r + H <= grid;
+    float ta = (float)q * fmaxf(1.0f, (float)grid / c);
+    if (can_split) ta += 0.5f * fmaxf(1.0f, (float)(2 * r) / c);
+    else if (r > 0) ta += fmaxf(1.0f, (float)r / c);
+    const int rounds = (F + grid - 1) / grid;
+    const int eff = rounds > 0 ? (F + rounds - 1) / rounds : grid;
+    const float tb = (float)rounds * fmaxf(1.0f, (float)eff / c);
+    if (F > 0 && tb < ta) {
+        sc.split = 0;
+        sc.ctas = eff;
+    } else {
+        sc.split = can_split ? r : 0;
+        sc.ctas = grid;
+    }
     sc.f_keep = F - sc.split;
-    sc.total = sc.f_keep + 2 * sc.split + n_pairs * sc.has_half;
+    sc.total = sc.f_keep + 2 * sc.split + H;
     return sc;
 }
 
@@ -373,7 +393,7 @@ __global__ void __launch_bounds__(kFThreads, 1) decode_ffn_kernel(const __grid_c
 
     const Sched sched = make_sched(early ? sc.P + (p.n_shared ? 1 : 0) : sc.n_pairs, p.I, (int)gridDim.x, early ? 1 : 0);
     const int total = sched.total;
-    const int w_begin = (int)blockIdx.x, w_stride = (int)gridDim.x;
+    const int w_begin = (int)blockIdx.x < sched.ctas ? (int)blockIdx.x : total, w_stride = sched.ctas;
     const uint32_t tmem_base = tmem_base_s;
     const int nkb = p.d / kFBK;
     volatile int* abort_flag = &abort_s;

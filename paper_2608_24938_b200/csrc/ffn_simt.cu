@@ -85,11 +85,12 @@ __global__ void combine_routes_kernel(const float* __restrict__ out, const float
 }
 
 // Eq. 4's weighted sum for the tensor-core path: GEMM-2 stored w~ * E(x) per route in bf16, sorted by
-// expert; a token's routes are found through the inverse permutation and summed in fp32, slot order.
+// expert; a token's routes are found through the inverse permutation and summed in fp32, slot order
+// (a decode step with a K split: the `parts` planes of a row, in order, inside that).
 __global__ void __launch_bounds__(256) combine_rows_kernel(const __nv_bfloat16* __restrict__ O,
                                                            const int32_t* __restrict__ inv_pos, int64_t Tn, int Kr, int d,
                                                            int n_shared, const int32_t* __restrict__ shared0_dev,
-                                                           __nv_bfloat16* __restrict__ y) {
+                                                           int parts, int64_t part_rows, __nv_bfloat16* __restrict__ y) {
     const int64_t i = blockIdx.x;
     grid_dep_launch();
     grid_dep_wait();
@@ -100,13 +101,15 @@ __global__ void __launch_bounds__(256) combine_rows_kernel(const __nv_bfloat16* 
             if (j == Kr && !n_shared) break;
             const int64_t row = j < Kr ? (int64_t)inv_pos[i * Kr + j] : shared0 + i;
             if (row < 0) continue;  // a slot merged into an earlier one of the same token
-            const uint4 v = *reinterpret_cast<const uint4*>(O + row * d + c);
-            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+            for (int part = 0; part < parts; ++part) {
+                const uint4 v = *reinterpret_cast<const uint4*>(O + (part * part_rows + row) * d + c);
+                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float2 f = __bfloat1622float2(h2[u]);
-                acc[2 * u] += f.x;
-                acc[2 * u + 1] += f.y;
+                for (int u = 0; u < 4; ++u) {
+                    const float2 f = __bfloat1622float2(h2[u]);
+                    acc[2 * u] += f.x;
+                    acc[2 * u + 1] += f.y;
+                }
             }
         }
         uint4 o;
@@ -194,9 +197,11 @@ cudaError_t launch_combine_routes(const float* out, const float* w, int64_t T, i
 }
 
 cudaError_t launch_combine_rows(const __nv_bfloat16* O, const int32_t* inv_pos, int64_t T, int Kr, int d,
-                                int n_shared, const int32_t* shared0_dev, __nv_bfloat16* y, cudaStream_t s) {
+                                int n_shared, const int32_t* shared0_dev, int parts, int64_t part_rows,
+                                __nv_bfloat16* y, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
-    return launch_pdl(combine_rows_kernel, (unsigned)T, 256, 0, s, O, inv_pos, T, Kr, d, n_shared, shared0_dev, y);
+    return launch_pdl(combine_rows_kernel, (unsigned)T, 256, 0, s, O, inv_pos, T, Kr, d, n_shared, shared0_dev, parts,
+                      part_rows, y);
 }
 
 }  // namespace exfold

@@ -173,7 +173,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     }
     ptx::tc_fence_after();
     const int nt = p.n_ntiles;
-    const int ks = (DEC && MODE == 1) ? p.ksplit : 1;  // K parts per tile (needs the fp32-reduction epilogue)
+    const int ks = (DEC && MODE == 1) ? p.ksplit : 1;  // K parts per tile (each part's rows go to a plane of their own)
     const int total = s_ws[G] * nt * ks;
     // Effective grid: with `rounds` items per CTA, ceil(total / rounds) CTAs finish together; the rest
     // stay idle instead of leaving a few CTAs one item behind (448 items on 148 SMs: 112 x 4, not
@@ -405,7 +405,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
 #pragma unroll
                             for (int j = 0; j < 16; ++j)
                                 pk[j] = pack_bf16(wv * __uint_as_float(v[2 * j]), wv * __uint_as_float(v[2 * j + 1]));
-                            const int64_t drow = p.store_rows ? grow : (int64_t)tok;
+                            // decode with a K split: part k of a row goes to plane k of the row buffer (p.R rows each)
+                            const int64_t drow = (p.store_rows ? grow : (int64_t)tok) + (DEC ? (int64_t)it.kpart * p.R : 0);
                             uint4* dst = reinterpret_cast<uint4*>(p.y + drow * p.d + col0);
 #pragma unroll
                             for (int j = 0; j < 4; ++j)

@@ -339,22 +339,32 @@ __global__ void __launch_bounds__(kDecThreads) decode_route_kernel(DecodeRoutePa
 
 
 // ---------------------------------------------------------------- token-parallel first half of decode routing
-// One CTA per token: (optionally) the router scores of Eq. 2 as fixed-order dot products - the same lane
-// partition, the same fused multiply-adds and the same shuffle tree as router_simt_kernel, so the scores are
-// those of exfold_router_logits bit for bit -, then the token's Top-K and its softmax weights in double
-// (slot order). CTA 0 also clears the status record.
-// The batch-level half (pool, targets, remap) runs in the prologue of the expert-FFN kernel (ffn_decode.cu).
-template <int NPL>
+// Per token: (optionally) the router scores of Eq. 2 as fixed-order dot products - the same lane partition, the
+// same fused multiply-adds and the same shuffle tree as router_simt_kernel, so the scores are those of
+// exfold_router_logits bit for bit -, then the token's Top-K and its softmax weights in double (slot order).
+// Without the router: one CTA per token. With it: a cluster of 8 CTAs per token, each taking an eighth of the
+// experts (one CTA alone would walk the whole router matrix with a handful of loads in flight); the scores meet
+// in the shared memory of the cluster's first CTA, which then ranks them. CTA 0 also clears the status record.
+// The batch-level half (pool, targets, remap) runs in the prologue of the gate/up kernel (ffn_decode.cu).
+constexpr int kTopkCluster = 8;
+
+template <int NPL, bool ROUTER>
 __global__ void __launch_bounds__(256) decode_topk_kernel(DecodeTopkParams p) {
     __shared__ float s_lg[kMaxExperts];
-    const int i = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int N = p.N, K = p.K, d = p.d;
+    const int i = ROUTER ? (int)blockIdx.x / kTopkCluster : (int)blockIdx.x;
     grid_dep_launch();
     grid_dep_wait();  // x may be the previous layer's output; the workspace may still be read by the previous call
-    if (i == 0 && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
-    if (p.w_router != nullptr) {
+    if (blockIdx.x == 0 && threadIdx.x < 4) reinterpret_cast<int*>(p.status)[threadIdx.x] = 0;
+    if (ROUTER) {
+        cg::cluster_group cluster = cg::this_cluster();
+        const int rank = (int)cluster.block_rank();
+        float* lead = cluster.map_shared_rank(s_lg, 0);
+        const int per = (N + kTopkCluster - 1) / kTopkCluster;
+        const int e_lo = rank * per, e_hi = min(N, e_lo + per);
         const __nv_bfloat16* xi = p.x + (size_t)i * d;
-        for (int e = warp; e < N; e += 8) {
+        for (int e = e_lo + warp; e < e_hi; e += 8) {
             const __nv_bfloat16* we = p.w_router + (size_t)e * d;
             float acc = 0.f;
             for (int c = lane * 8; c < d; c += 256) {
@@ -371,18 +381,19 @@ __global__ void __launch_bounds__(256) decode_topk_kernel(DecodeTopkParams p) {
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
             if (lane == 0) {
-                s_lg[e] = acc;
+                lead[e] = acc;
                 p.logits_out[(size_t)i * N + e] = acc;
             }
         }
-        __syncthreads();
+        cluster.sync();  // every score of the token is in the first CTA's shared memory
+        if (rank != 0) return;
     }
     if (warp != 0) return;
     float v[NPL];
 #pragma unroll
     for (int q = 0; q < NPL; ++q) {
         const int e = lane + 32 * q;
-        v[q] = e < N ? (p.w_router != nullptr ? s_lg[e] : p.logits[(size_t)i * N + e]) : -INFINITY;
+        v[q] = e < N ? (ROUTER ? s_lg[e] : p.logits[(size_t)i * N + e]) : -INFINITY;
     }
     uint32_t key_q[NPL];
     uint32_t used = 0;
@@ -495,11 +506,20 @@ cudaError_t launch_decode_route(const DecodeRouteParams& p, cudaStream_t s) {
 
 cudaError_t launch_decode_topk(const DecodeTopkParams& p, cudaStream_t s) {
     const int npl = (p.N + 31) / 32;
+    if (p.w_router != nullptr) {
+        const unsigned grid = (unsigned)p.B * kTopkCluster;
+        switch (npl) {
+            case 1: return launch_pdl_cluster(decode_topk_kernel<1, true>, grid, 256, 0, kTopkCluster, s, p);
+            case 2: return launch_pdl_cluster(decode_topk_kernel<2, true>, grid, 256, 0, kTopkCluster, s, p);
+            case 3: case 4: return launch_pdl_cluster(decode_topk_kernel<4, true>, grid, 256, 0, kTopkCluster, s, p);
+            default: return launch_pdl_cluster(decode_topk_kernel<8, true>, grid, 256, 0, kTopkCluster, s, p);
+        }
+    }
     switch (npl) {
-        case 1: return launch_pdl(decode_topk_kernel<1>, p.B, 256, 0, s, p);
-        case 2: return launch_pdl(decode_topk_kernel<2>, p.B, 256, 0, s, p);
-        case 3: case 4: return launch_pdl(decode_topk_kernel<4>, p.B, 256, 0, s, p);
-        default: return launch_pdl(decode_topk_kernel<8>, p.B, 256, 0, s, p);
+        case 1: return launch_pdl(decode_topk_kernel<1, false>, p.B, 256, 0, s, p);
+        case 2: return launch_pdl(decode_topk_kernel<2, false>, p.B, 256, 0, s, p);
+        case 3: case 4: return launch_pdl(decode_topk_kernel<4, false>, p.B, 256, 0, s, p);
+        default: return launch_pdl(decode_topk_kernel<8, false>, p.B, 256, 0, s, p);
     }
 }
 
