@@ -368,13 +368,19 @@ def decode_roofline(wl, kern, peaks, pool):
     cfg = wl.cfg
     byts = (pool + cfg.n_shared) * 3.0 * cfg.hidden * cfg.inter * wl.el
     name = cfg.name.replace("-reduced", "")
-    if "decode_ffn" in kern:  # one fused kernel streams gate, up and down weights
+    if "decode_ffn" in kern:  # gate/up kernel (routing prologue + the pool's gate and up weights, x read in place)
+        gu = byts * 2.0 / 3.0
         t = kern["decode_ffn"] * 1e-3
         ratio = NCU_TRAFFIC_RATIO.get(name, {}).get("decode_ffn")
-        return {"kernel": "decode fused expert FFN (gate/up/down weight stream over the pool), tcgen05", "bound": "hbm",
-                "achieved": r4(byts / t / 1e9), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": r4(byts / t / 1e9 / peaks["hbm_gbs"]), "traffic": None if ratio is None else byts * ratio,
-                "bytes_per_launch": byts, "launch_ms": r4(kern["decode_ffn"])}
+        out = {"kernel": "decode gate/up kernel (pool / remap prologue + gate and up weight stream over the pool), tcgen05",
+               "bound": "hbm", "achieved": r4(gu / t / 1e9), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+               "frac": r4(gu / t / 1e9 / peaks["hbm_gbs"]), "traffic": None if ratio is None else gu * ratio,
+               "bytes_per_launch": gu, "launch_ms": r4(kern["decode_ffn"])}
+        td = kern.get("decode_down", 0.0) * 1e-3
+        if td > 0:
+            out["down_gbs"] = r4(byts / 3.0 / td / 1e9)
+            out["ffn_gbs"] = r4(byts / (t + td) / 1e9)
+        return out
     if "decode_gateup" in kern:
         gu = byts * 2.0 / 3.0
         tg = kern["decode_gateup"] * 1e-3
@@ -427,7 +433,7 @@ def cpu_baseline_leg(wl, Kp, M, flop_budget):
     cfg = wl.cfg
     d, I, K = cfg.hidden, cfg.inter, cfg.top_k
     per_tok = (Kp + cfg.n_shared) * 6.0 * d * I
-    n_s = int(max(1, min(256, flop_budget / per_tok)))
+    n_s = int(max(1, min(2048, flop_budget / per_tok)))
     t0 = time.time()
     o = oracle_sample_run(cfg, wl.inp, Kp, n_s)
     yg = wl.y.float().cpu().numpy()[o["idx"]]
@@ -815,7 +821,7 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-sustained", action="store_true")
     ap.add_argument("--skip-configs", action="store_true")
-    ap.add_argument("--cpu-flop-budget", type=float, default=3e11,
+    ap.add_argument("--cpu-flop-budget", type=float, default=3e12,
                     help="flop of oracle work in the cpu-baseline sample (about 10-30 s of CPU time)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
