@@ -56,6 +56,7 @@ struct Scratch {  // per-batch routing state, one copy per CTA
     int pool[kMaxExperts];     // pool experts by rank
     int target[kMaxExperts];
     float scale[kMaxExperts];
+    float h[kMaxExperts];      // norm table (dynamic pool), staged before the dependency wait
     int cnt[kFMaxPairs];       // rows of (group, token tile): distinct tokens of the tile that the group serves
     int goff[kFMaxPairs + 2];  // exclusive prefix of cnt: first compact row of (group, token tile)
     int pairs[kFMaxPairs];     // the pairs that have rows, in order: group * 2 + token tile
@@ -188,7 +189,8 @@ __global__ void __launch_bounds__(kFThreads, 1) decode_ffn_kernel(const __grid_c
         sc.rank_of[e] = -1;
     }
     for (int i = threadIdx.x; i < kFMaxPairs; i += kFThreads) sc.cnt[i] = 0;
-    if (!is_static) {  // warm L2 with the loss and scalar tables while the previous kernel still runs
+    if (!is_static) {  // the norm table into shared memory, the loss and scalar tables into L2, while the previous kernel runs
+        for (int e = threadIdx.x; e < N; e += kFThreads) sc.h[e] = __ldg(p.h + e);
         const size_t n_el = (size_t)N * N, lines = (n_el * 4 + 127) / 128;
         for (size_t i = (size_t)blockIdx.x * kFThreads + threadIdx.x; i < lines; i += (size_t)gridDim.x * kFThreads) {
             const size_t el = i * 32 < n_el ? i * 32 : n_el - 1;
@@ -235,24 +237,25 @@ __global__ void __launch_bounds__(kFThreads, 1) decode_ffn_kernel(const __grid_c
                 const unsigned long long acc = (unsigned long long)sc.acc32[3 * e] +
                                                ((unsigned long long)sc.acc32[3 * e + 1] << 21) +
                                                ((unsigned long long)sc.acc32[3 * e + 2] << 42);
-                const double score = (double)acc * (1.0 / 9007199254740992.0) * (double)p.h[e] + 0.0;
+                const double score = (double)acc * (1.0 / 9007199254740992.0) * (double)sc.h[e] + 0.0;
                 key = __double_as_longlong(score);
                 if (key < 0) key ^= 0x7FFFFFFFFFFFFFFFll;  // negative doubles: larger magnitude = smaller
             }
             sc.key[e] = key;
         }
         __syncthreads();
-        // pool = best min(M, |U|) experts of the union by (score desc, id asc): rank by counting, a thread per expert
-        for (int e = threadIdx.x; e < N; e += kFThreads) {
+        // pool = best min(M, |U|) experts of the union by (score desc, id asc): rank by counting, a warp per expert
+        // (integer compares on the keys: the lanes split the other experts, one hardware reduction adds them up)
+        for (int e = warp; e < N; e += kFThreads / 32) {
             const long long ke = sc.key[e];
-            if (ke == LLONG_MIN) continue;
+            if (ke == LLONG_MIN) continue;  // warp-uniform
             int better = 0;
-#pragma unroll 8
-            for (int o = 0; o < N; ++o) {
-                const long long ko = sc.key[o];  // the same address in every lane: a broadcast
+            for (int o = lane; o < N; o += 32) {
+                const long long ko = sc.key[o];
                 better += (ko > ke || (ko == ke && o < e)) ? 1 : 0;
             }
-            if (better < p.M) {
+            better = __reduce_add_sync(0xffffffffu, better);
+            if (lane == 0 && better < p.M) {
                 sc.rank_of[e] = better;
                 sc.pool[better] = e;
             }
