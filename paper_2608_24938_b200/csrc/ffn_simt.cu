@@ -129,12 +129,11 @@ __global__ void __launch_bounds__(256) combine_rows_kernel(const __nv_bfloat16* 
                         if (row[u] >= 0) add(v[u]);
                 }
             }
-        } else {
-            for (int j = 0; j < n_src; ++j) {
+        } else {  // prefill: every slot has a row of its own and there is one plane
+            for (int j = 0; j <= Kr; ++j) {
+                if (j == Kr && !n_shared) break;
                 const int64_t row = j < Kr ? (int64_t)inv_pos[i * Kr + j] : shared0 + i;
-                if (row < 0) continue;
-                for (int part = 0; part < parts; ++part)
-                    add(*reinterpret_cast<const uint4*>(O + (part * part_rows + row) * d + c));
+                add(*reinterpret_cast<const uint4*>(O + row * d + c));
             }
         }
         uint4 o;
@@ -225,7 +224,7 @@ cudaError_t launch_combine_rows(const __nv_bfloat16* O, const int32_t* inv_pos, 
                                 int n_shared, const int32_t* shared0_dev, int parts, int64_t part_rows,
                                 __nv_bfloat16* y, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
-    if (T <= 1024)
+    if (T <= 1024 || parts > 1 || shared0_dev != nullptr)  // decode (merged slots are marked -1, K planes)
         return launch_pdl(combine_rows_kernel<true>, (unsigned)T, 256, 0, s, O, inv_pos, T, Kr, d, n_shared, shared0_dev,
                           parts, part_rows, y);
     return launch_pdl(combine_rows_kernel<false>, (unsigned)T, 256, 0, s, O, inv_pos, T, Kr, d, n_shared, shared0_dev, parts,
