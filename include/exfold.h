@@ -211,8 +211,12 @@ int exfold_moe_prefill_ex(const exfold_layer *layer, const void *x, const float 
  * Decode: batch-level expert-pool folding (Eq. 11, 12, 14, then Eq. 1 and 4 over the pool
  * only). x [B][d], logits [B][N] -> y [B][d], B <= 256. pool_m = M in [1, N]; the pool is
  * the whole expert union of the batch when that has at most M experts, so pool_m = N is the
- * unfolded layer. Scores are accumulated in double, tokens ascending. Only the pool's (and
- * the shared expert's) weights are read.
+ * unfolded layer. Scores are sums of the double-precision routed weights (exact in 2^-53 fixed
+ * point, so independent of any order). Only the pool's (and the shared expert's) weights are
+ * read, each byte once. bf16 layers: four kernels chained by programmatic dependent launch
+ * (per-token Top-K; gate/up projection with the batch-level routing in its prologue, x read in
+ * place; grouped down projection over one row per distinct (token, pool expert); per-token sum
+ * of those rows in slot order). No atomics are used: the same inputs give the same bits.
  */
 int exfold_moe_decode(const exfold_layer *layer, const void *x, const float *logits, int64_t B,
                       const void *w_gate, const void *w_up, const void *w_down,
