@@ -107,6 +107,22 @@ def test_bad_arguments_are_rejected_before_launch(ex):
     assert router(ws=p + 8) == ex.EXFOLD_ERR_INVALID_ARG
     assert router(wsb=64) == ex.EXFOLD_ERR_WORKSPACE_TOO_SMALL
 
+    def dec_layer(wr=p, lg=p, B=4, wsb=big):
+        return ex.lib.exfold_moe_decode_layer(C.byref(layer), p, wr, B, p, p, p, C.byref(tabs), 2, lg, p, None, p, wsb, None)
+
+    def pre_layer(kp=1, T=4, wsb=big):
+        return ex.lib.exfold_moe_prefill_layer(C.byref(layer), p, p, T, p, p, p, C.byref(tabs), kp, p, p, None, p, wsb, None)
+
+    assert dec_layer(wr=None) == ex.EXFOLD_ERR_INVALID_ARG
+    assert dec_layer(lg=None) == ex.EXFOLD_ERR_INVALID_ARG
+    assert dec_layer(lg=p + 4) == ex.EXFOLD_ERR_INVALID_ARG    # scores buffer not 16-byte aligned
+    assert dec_layer(B=0) == ex.EXFOLD_ERR_INVALID_ARG
+    assert dec_layer(B=257) == ex.EXFOLD_ERR_UNSUPPORTED
+    assert dec_layer(wsb=1024) == ex.EXFOLD_ERR_WORKSPACE_TOO_SMALL
+    assert pre_layer(kp=3) == ex.EXFOLD_ERR_INVALID_ARG
+    assert pre_layer(wsb=1024) == ex.EXFOLD_ERR_WORKSPACE_TOO_SMALL
+    assert ex.lib.exfold_static_scratch_address(None) == ex.EXFOLD_ERR_INVALID_ARG
+
 
 def test_product_package_does_not_touch_the_oracle():
     """The CUDA path and the oracle share no code and neither imports the other."""
