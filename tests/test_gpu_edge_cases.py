@@ -189,3 +189,38 @@ def test_two_prefill_calls_on_two_streams_of_one_thread():
                           wss[0])
     assert ex.exfold_device_status(wss[0]) == 0
     assert np.array_equal(ys[0].float().cpu().numpy(), y_ref)
+
+
+# ------------------------------------------------------------------ layer calls (router matrix in) on an fp32 layer
+def test_layer_calls_on_an_fp32_layer():
+    """fp32 layers take the separate dot-product router kernel and the SIMT expert path behind the same entry points."""
+    cfg = si.CONFIGS["tiny"]
+    case = Case(cfg)
+    ex, dev = case.ex, case.dev
+    T, B, K, N = case.T, case.B, cfg.top_k, cfg.n_experts
+    wr = si.router_weights(cfg, std=2.0 / np.sqrt(cfg.hidden))
+    S, L, h, lnh = case.np_tables()
+    ws = case.workspace(max(T, B), K)
+    for x, d_x, n, decode in ((case.x, case.d_x, T, False), (case.xd, case.d_xd, B, True)):
+        r32, r64 = oracle.router_logits(A(x), A(wr))
+        srt = np.sort(r64, axis=1)[:, ::-1]
+        assert (srt[:, :K] - srt[:, 1:K + 1]).min() > 1e-4, "seeded scores without near-ties"
+        lg = torch.full((n, N), float("nan"), device=dev)
+        y = torch.full((n, cfg.hidden), float("nan"), dtype=torch.float32, device=dev)
+        i32 = dict(dtype=torch.int32, device=dev)
+        if decode:
+            meta = dict(ids=torch.full((n, K), -7, **i32))
+            ex.exfold_moe_decode_layer(case.layer, d_x, wr.to(dev), case.d_wg, case.d_wu, case.d_wd, case.tables, 4, y,
+                                       ws, logits_out=lg, meta=meta)
+            ref = oracle.decode_fold(r32, K, 4, S, L, h)
+        else:
+            meta = dict(ids=torch.full((n, 1), -7, **i32))
+            ex.exfold_moe_prefill_layer(case.layer, d_x, wr.to(dev), case.d_wg, case.d_wu, case.d_wd, case.tables, 1, y,
+                                        ws, logits_out=lg, meta=meta)
+            ref = oracle.prefill_fold(r32, K, 1, S, L, h, lnh)
+        assert ex.exfold_device_status(ws) == 0
+        assert np.abs(lg.cpu().numpy() - r32).max() <= 1e-5 * np.abs(r32).max()
+        assert np.array_equal(meta["ids"].cpu().numpy(), ref["ids"])
+        yref = oracle.moe_apply(A(x), A(case.wg), A(case.wu), A(case.wd), ref["ids"], ref["w"], N, cfg.n_shared)
+        # the weights come from scores that differ in the last bits: looser than the same-logits fp32 bound
+        assert np.abs(y.cpu().numpy() - yref).max() <= 1e-3 * np.abs(yref).max()
