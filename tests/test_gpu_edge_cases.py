@@ -224,3 +224,27 @@ def test_layer_calls_on_an_fp32_layer():
         yref = oracle.moe_apply(A(x), A(case.wg), A(case.wu), A(case.wd), ref["ids"], ref["w"], N, cfg.n_shared)
         # the weights come from scores that differ in the last bits: looser than the same-logits fp32 bound
         assert np.abs(y.cpu().numpy() - yref).max() <= 1e-3 * np.abs(yref).max()
+
+
+# ------------------------------------------------------------------ a long prompt: many super-blocks of route blocks
+@pytest.mark.parametrize("T,kw", [(150_001, dict(n_experts=8, top_k=2, k_pre=(1,), hidden=64, inter=64)),
+                                  (70_000, dict(n_experts=40, n_shared=1, top_k=4, k_pre=(2,), hidden=64, inter=128))])
+def test_long_prompt_sorted_routes(T, kw):
+    """The sorted position of a route is (rows of lower experts) + (rows of its expert in earlier route blocks);
+    the scatter kernel takes both from two levels of histograms (per block of 32 tokens, per super-block of 64 blocks).
+    150 001 tokens are 4688 blocks in 74 super-blocks with a ragged last block: permutation, offsets and retained
+    experts bit-exact against the oracle's stable sort, outputs on a token sample."""
+    case = Case(small_bf16(prefill_tokens=T, decode_batch=8, logits="zipf", **kw), std=0.2)
+    cfg, Kp = case.cfg, case.cfg.k_pre[0]
+    got = case.run_prefill(Kp)
+    S, L, h, lnh = case.np_tables()
+    ref = oracle.prefill_fold(case.lg.numpy(), cfg.top_k, Kp, S, L, h, lnh)
+    perm, off = oracle.sort_routes(ref["ids"], cfg.n_experts)
+    assert np.array_equal(got["ids"], ref["ids"])
+    assert np.array_equal(got["offsets"], off)
+    assert np.array_equal(got["perm"], perm)
+    idx = np.concatenate([sample_tokens(T, 48), np.array([0, T - 1])])
+    idx = np.unique(idx)
+    yref = oracle.moe_apply(A(case.x), A(case.wg), A(case.wu), A(case.wd), ref["ids"], ref["w"], cfg.n_experts,
+                            cfg.n_shared, tok_idx=idx)
+    check_output(got["y"][idx], yref, "bf16")
