@@ -22,8 +22,8 @@
  *     workspace `ws` (exfold_workspace_bytes; 256-byte aligned). Calls that share a
  *     workspace must be ordered on one stream.
  *   - What the library keeps between calls, and nothing else: (a) per host thread and device,
- *     created on first use and freed by exfold_thread_release: one extra CUDA stream with three
- *     events (large prefill calls run two kernel chains side by side on it) and two copy streams
+ *     created on first use and freed by exfold_thread_release: one extra CUDA stream (highest priority) with
+ *     three events (large prefill calls run two kernel chains side by side on it) and two copy streams
  *     with ten events (chunked host-buffer prefill). Calls issued by one host thread on
  *     different caller streams share them, so the parts that use them run one after the other;
  *     results do not depend on it. (b) per process: the launch counter, the optional
@@ -171,9 +171,11 @@ int exfold_calibrate_layers(const exfold_layer *layer, const exfold_calib_job *j
  * bf16 layers: the two grouped GEMMs of a call of >= 24 row tiles (128 sorted rows each) run the experts' row tiles
  * two at a time on pairs of CTAs and, beside them, the experts' odd last tiles on the one-CTA-per-tile kernel;
  * smaller calls use the latter alone. The results are bit-identical either way. The odd-tile kernels run on a
- * second stream that the library creates once per host thread; they are ordered after the caller's earlier work and
- * before its later work by events on the caller's stream (also under stream capture). exfold_fold_opts.gemm_path
- * overrides the choice of kernels (tests and measurements).
+ * second stream (highest priority) that the library creates once per host thread; with a shared expert, the gate/up
+ * projection of its whole row-tile pairs also runs there, beside the kernel that gathers the routed rows (its inputs
+ * are x and the weights only). That work is ordered after the caller's earlier work and before its later work by
+ * events on the caller's stream (also under stream capture). exfold_fold_opts.gemm_path overrides the choice of
+ * kernels (tests and measurements).
  */
 int exfold_moe_prefill(const exfold_layer *layer, const void *x, const float *logits, int64_t T,
                        const void *w_gate, const void *w_up, const void *w_down,

@@ -202,9 +202,14 @@ bool new_event(cudaEvent_t* e) { return cudaEventCreateWithFlags(e, cudaEventDis
 // second stream (and fork / join events) for the odd-tile passes of a prefill call
 ThreadDeviceState* side_stream() {
     ThreadDeviceState* h = thread_state();
-    if (h && !h->side_ok)
-        h->side_ok = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) == cudaSuccess && new_event(&h->fork) &&
-                     new_event(&h->join) && new_event(&h->mid);
+    if (h && !h->side_ok) {
+        // highest priority: what runs here beside a bandwidth-bound kernel of the caller's stream (the shared
+        // expert's GEMM-1 beside the scatter kernel) gets its SMs first and the other kernel fills the rest
+        int lo = 0, hi = 0;
+        if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) hi = 0;
+        h->side_ok = cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, hi) == cudaSuccess &&
+                     new_event(&h->fork) && new_event(&h->join) && new_event(&h->mid);
+    }
     return h && h->side_ok ? h : nullptr;
 }
 // copy-in / copy-out streams and events of the chunked host-buffer prefill
@@ -419,6 +424,30 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
     rp.status = t_keep_status ? nullptr : at<DeviceStatus>(ws, pl.status);
     { ProfScope ps(0, s); EXFOLD_CUDA(launch_prefill_route(rp, s)); }
 
+    // The shared expert's gate/up projection needs nothing the routing kernels produce (its rows are x itself, its
+    // rows of H lie behind the routed ones): its whole row-tile pairs run on the second stream beside the scatter
+    // kernel, which moves bytes while the tensor pipes would idle. (After the routing kernel, which clears the status
+    // record every kernel's waits look at.) The CTA-pair GEMM-1 that follows the scatter kernel skips those pairs.
+    // Not with per-kernel timing on: the timed kernels are then the plain sequence, GEMM-1 with all its pairs.
+    const int shared_pairs = pairs && l.n_shared && !g_prof.on ? (int)(((T + kTileM - 1) / kTileM) / 2) : 0;
+    ThreadDeviceState* early_side = nullptr;
+    if (shared_pairs > 0) {
+        early_side = side_stream();
+        if (!early_side) return EXFOLD_ERR_CUDA;
+        GroupedGemmParams gs{};
+        gs.tm_a = tm_xs; gs.tm_a2 = tm_x; gs.tm_b0 = tm_wg; gs.tm_b1 = tm_wu; gs.x_rows = (int)T;
+        gs.G = G; gs.n_routed = N; gs.R = (int)R; gs.d = d; gs.I = I; gs.n_ntiles = (I + 127) / 128; gs.ksplit = 1;
+        gs.a_rows = kTileM; gs.H = at<__nv_bfloat16>(ws, pl.H); gs.status = at<DeviceStatus>(ws, pl.status);
+        gs.shared_split = 1;
+        gs.sbs = SideBySide{(I + 127) / 128, d / kGemmBK, (d + 255) / 256, I / kGemmBK, sms / 2, 0, 0};
+        EXFOLD_CUDA(cudaEventRecord(early_side->fork, s));
+        EXFOLD_CUDA(cudaStreamWaitEvent(early_side->side, early_side->fork, 0));
+        EXFOLD_CUDA(launch_grouped_gemm1_pair(gs, sms, early_side->side));
+        EXFOLD_CUDA(cudaEventRecord(early_side->mid, early_side->side));
+    }
+    SideJoin early_join{early_side, s};  // joins the second stream on the error returns before the passes below take over
+    early_join.armed = early_side != nullptr;
+
     PrefillScatterParams cp{};
     cp.T = T; cp.N = N; cp.n_shared = l.n_shared; cp.Kp = Kp; cp.d_bytes = bf16 ? d * 2 : 0;
     cp.nblk = (int)((T + kRouteTokensPerBlock - 1) / kRouteTokensPerBlock);
@@ -468,11 +497,16 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
             const double odd_est = std::max<double>(1.0, G / 2.0), pair_est = std::max<double>(1.0, (tiles_est - G / 2.0) / 2.0);
             const double q_est = sms * odd_est / (odd_est + 2 * 0.73 * pair_est);
             const int odd_grid = std::min(sms, 2 * (int)std::ceil(q_est) + 8) & ~1;
-            const SideBySide sbs{nt1, d / kGemmBK, nt2, I / kGemmBK, sms / 2, odd_grid};
+            const SideBySide sbs{nt1, d / kGemmBK, nt2, I / kGemmBK, sms / 2, odd_grid, shared_pairs};
             g.sbs = g2.sbs = go1.sbs = go2.sbs = sbs;
+            if (shared_pairs > 0) {  // the shared expert's pairs of GEMM-1 are done (or running) on the second stream
+                g.shared_split = 2;
+                EXFOLD_CUDA(cudaStreamWaitEvent(s, side.mid, 0));
+            }
             EXFOLD_CUDA(cudaEventRecord(side.fork, s));
             EXFOLD_CUDA(cudaStreamWaitEvent(side.side, side.fork, 0));
             SideJoin joiner{sidep, s};
+            early_join.armed = false;
             {
                 ProfScope ps(3, s);
                 { ProfScope pp(12, s); EXFOLD_CUDA(launch_grouped_gemm1_pair(g, sms, s)); }

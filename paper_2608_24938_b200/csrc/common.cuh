@@ -323,6 +323,8 @@ struct SideBySide {
     int nt1, nkb1, nt2, nkb2;  // column tiles and k-blocks per work item of GEMM-1 and GEMM-2
     int n_sm_pairs;            // SM pairs the pair passes are launched over
     int odd_ctas;              // CTAs the odd-tile passes are launched with (even); 0: the passes do not run side by side
+    int shared_pairs1;         // whole row-tile pairs of the shared expert that GEMM-1's pair pass does not run (they
+                               // ran beside the routing kernels, GroupedGemmParams::shared_split), else 0
 };
 __host__ __device__ inline int pair_pass_clusters(int pairs, int odd, const SideBySide& sb) {
     const int n = sb.n_sm_pairs;
@@ -333,7 +335,8 @@ __host__ __device__ inline int pair_pass_clusters(int pairs, int odd, const Side
     float best_t = 3.0e38f;
     for (int P = best; P < n; ++P) {
         const int Q = 2 * (n - P);
-        const float tp = 0.73f * (float)(((pairs * sb.nt1 + P - 1) / P) * sb.nkb1 + ((pairs * sb.nt2 + P - 1) / P) * sb.nkb2);
+        const int pairs1 = pairs - sb.shared_pairs1;
+        const float tp = 0.73f * (float)(((pairs1 * sb.nt1 + P - 1) / P) * sb.nkb1 + ((pairs * sb.nt2 + P - 1) / P) * sb.nkb2);
         const float to = (float)(((odd * sb.nt1 + Q - 1) / Q) * sb.nkb1 + ((odd * sb.nt2 + Q - 1) / Q) * sb.nkb2);
         const float t = tp > to ? tp : to;
         if (t < best_t) {
@@ -368,6 +371,9 @@ struct GroupedGemmParams {
     int store_rows;             // 1: y is the per-route buffer O[row][d] that the combine kernel sums
     float* o32;                 // GEMM-2, calibration: unweighted fp32 outputs O32[row][d] (null: the epilogues above)
     int x_rows;                 // GEMM-1: rows of x; a group that reads x directly starts at row (row0 - R) % x_rows
+    int shared_split;           // CTA-pair GEMM-1. 1: this launch runs only the whole row-tile pairs of the shared expert
+                                //    (rows [R, R + x_rows) of expert n_routed, read from x: nothing the routing kernels
+                                //    write is touched, so it runs beside them); 2: those pairs ran that way, skip them
     int odd_only;               // 1: only each group's last row tile, and only if its tile count is odd (the rest ran on CTA pairs)
     SideBySide sbs;             // odd_ctas > 0: the CTA-pair pass and the odd-tile pass run at the same time (two
                                 //    streams); each keeps its share of the SM pairs (pair_pass_clusters) and the CTAs

@@ -38,7 +38,7 @@ struct PairItem {
     int g, row0, rows1, n_idx;  // rows1: valid rows of the second tile (the first is always full)
 };
 
-// Work index -> (group, column tile, pair of row tiles); order: group, column tile, pair (fastest)
+// Work index -> (group, column tile, pair of row tiles); order: group, then see below
 __device__ __forceinline__ PairItem decode_pair(int w, int G, int nt, const int* s_off, const int* s_wp) {
     int lo = 0, hi = G;
     while (hi - lo > 1) {
@@ -51,8 +51,12 @@ __device__ __forceinline__ PairItem decode_pair(int w, int G, int nt, const int*
     it.g = lo;
     const int pairs = s_wp[lo + 1] - s_wp[lo];
     const int local = w - s_wp[lo] * nt;
-    const int j = local % pairs;
-    it.n_idx = local / pairs;
+    // Within a group the faster index is the one with fewer values: clusters that run together then share the
+    // larger operand through L2 (few pairs: they share a weight tile and each re-reads its rows per column tile;
+    // more pairs than column tiles, e.g. a shared expert that sees every token: they share rows and re-read weights)
+    const bool rows_outer = pairs > nt;
+    const int j = rows_outer ? local / nt : local % pairs;
+    it.n_idx = rows_outer ? local - j * nt : local / pairs;
     it.row0 = s_off[lo] + j * 2 * kTileM;
     const int left1 = s_off[lo + 1] - it.row0 - kTileM;
     it.rows1 = left1 < kTileM ? left1 : kTileM;
@@ -108,8 +112,11 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
         ptx::tmem_relinquish_pair();
     }
     grid_dep_wait();  // everything below reads what the routing kernels (or GEMM-1) wrote
-    const int G = p.G;
-    for (int i = threadIdx.x; i <= G; i += kPThreads) s_off[i] = p.offsets[i];
+    // shared_split == 1: one group, the shared expert's rows; the offsets table is not read (the kernel that writes it
+    // may still be running)
+    const bool shared_only = MODE == 0 && p.shared_split == 1;
+    const int G = shared_only ? 1 : p.G;
+    for (int i = threadIdx.x; i <= G; i += kPThreads) s_off[i] = shared_only ? p.R + i * p.x_rows : p.offsets[i];
     ptx::tc_fence_before();
     __syncthreads();
     if (warp == 0) {  // prefix of whole row-tile pairs per group, 32 groups per step
@@ -119,7 +126,7 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
             int pairs = 0;
             if (g < G) {
                 const int tiles = (s_off[g + 1] - s_off[g] + kTileM - 1) / kTileM;
-                pairs = tiles >> 1;
+                pairs = (MODE == 0 && p.shared_split == 2 && g == p.n_routed) ? 0 : tiles >> 1;
                 odd += tiles & 1;
             }
             int incl = pairs;
@@ -143,7 +150,9 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
     // beside the odd-tile pass this pass keeps only its share of the SM pairs; the other clusters leave at once
     // (both CTAs of a cluster take the same decision: nothing allocated, no cluster barrier entered)
     const bool side = p.sbs.odd_ctas > 0;
-    const int n_pairs = side ? pair_pass_clusters(s_wp[G], s_n_odd, p.sbs) : n_launched;
+    // (the split is taken on ALL pairs, in every kernel of the two passes alike; it discounts the skipped ones itself)
+    const int skipped = MODE == 0 && p.shared_split == 2 ? p.sbs.shared_pairs1 : 0;
+    const int n_pairs = side ? pair_pass_clusters(s_wp[G] + skipped, s_n_odd, p.sbs) : n_launched;
     const int rounds = n_pairs > 0 ? (total + n_pairs - 1) / n_pairs : 0;
     const int eff = rounds > 0 ? (total + rounds - 1) / rounds : 0;  // pairs that take work and finish together
     const int w_begin = pair_id < eff ? pair_id : total;
@@ -171,7 +180,7 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
             bool ok = true;
             for (int w = w_begin; w < total && ok; w += w_stride) {
                 const PairItem it = decode_pair(w, G, nt, s_off, s_wp);
-                const int expert = it.g;
+                const int expert = shared_only ? p.n_routed : it.g;
                 const bool from_x = MODE == 0 && expert >= p.n_routed;  // rows read from x itself, no gathered copy
                 const CUtensorMap* tma_a = from_x ? &p.tm_a2 : &p.tm_a;
                 const int arow = (from_x ? (it.row0 - p.R) % p.x_rows : it.row0) + rank * kTileM;

@@ -248,3 +248,35 @@ def test_long_prompt_sorted_routes(T, kw):
     yref = oracle.moe_apply(A(case.x), A(case.wg), A(case.wu), A(case.wd), ref["ids"], ref["w"], cfg.n_experts,
                             cfg.n_shared, tok_idx=idx)
     check_output(got["y"][idx], yref, "bf16")
+
+
+# ------------------------------------------------------------------ shared expert beside the scatter kernel, under capture
+def test_shared_expert_pairs_under_graph_capture():
+    """With a shared expert and enough rows for the CTA-pair kernels, the shared expert's gate/up pairs run on the
+    library's second stream beside the scatter kernel, and the odd-tile passes fork there a second time. The same
+    call captured into a CUDA graph (both forks and joins become graph edges) and replayed gives the bits of the
+    plain stream call; outputs against the oracle on a token sample."""
+    case = Case(small_bf16(n_shared=1, prefill_tokens=3001, hidden=256, inter=384, logits="normal"), std=0.1)
+    cfg, ex, dev = case.cfg, case.ex, case.dev
+    T, Kp = case.T, 2
+    ref = case.run_prefill(Kp, with_meta=False)["y"]
+    ws = case.workspace(T, Kp)
+    y = torch.full((T, cfg.hidden), float("nan"), dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        ex.exfold_moe_prefill(case.layer, case.d_x, case.d_lg, case.d_wg, case.d_wu, case.d_wd, case.tables, Kp, y, ws,
+                              stream=stream)   # warm-up outside the capture: the second stream is created here
+        stream.synchronize()
+        y.fill_(float("nan"))
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            ex.exfold_moe_prefill(case.layer, case.d_x, case.d_lg, case.d_wg, case.d_wu, case.d_wd, case.tables, Kp, y,
+                                  ws, stream=stream)
+        for _ in range(3):
+            graph.replay()
+        stream.synchronize()
+        assert ex.exfold_device_status(ws, stream) == 0
+    got = y.float().cpu().numpy()
+    assert np.array_equal(got, ref)
+    idx = sample_tokens(T, 40)
+    check_output(got[idx], case.oracle_prefill(Kp, tok_idx=idx)["y"], "bf16")
