@@ -49,9 +49,9 @@ NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}  # the figures the task sta
 # the full-size algorithmic bytes. A shape without a capture reports traffic = null.
 NCU_TRAFFIC_RATIO = {
     # profiles/kernels_mixtral_reduced.md, kernels_qwen3_full.md, kernels_glm45air_reduced.md
-    "mixtral": {"gemm1": 424.5 / 318.8, "decode_ffn": 138.2 / 134.7},
-    "qwen3": {"gemm1": 901.4 / 820.0, "decode_ffn": 104.0 / 101.7},
-    "glm45air": {"gemm1": 1346.7 / 986.7, "decode_ffn": 771.6 / 765.6},
+    "mixtral": {"gemm1": 426.8 / 318.8, "decode_ffn": 138.6 / 134.7},
+    "qwen3": {"gemm1": 899.7 / 820.0, "decode_ffn": 105.0 / 101.7},
+    "glm45air": {"gemm1": 1343.2 / 986.7, "decode_ffn": 771.6 / 765.6},
 }
 
 
