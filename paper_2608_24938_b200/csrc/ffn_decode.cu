@@ -78,7 +78,7 @@ struct Sched {  // the same in every role of a CTA
 //   (a) all CTAs, the last partial round of r full items cut into 2r halves when every half finds its own SM;
 //   (b) only eff = ceil(F / rounds) CTAs, each exactly `rounds` items, so that all of them finish together.
 // In units of the time one SM needs for a full item alone, a phase of n SMs working at once takes z * max(1, n / c)
-// for items of size z: about c = 110 streaming SMs saturate HBM (measured: ~55 GB/s per SM, ~6 TB/s together).
+// for items of size z: about c = 110 SMs of this kernel saturate HBM (measured: it streams ~55 GB/s per SM, ~6 TB/s together).
 // (b) wins when the remainder would leave a few SMs working alone (448 items: 112 x 4 rather than 148 x 3 + 8 halves).
 __device__ __forceinline__ Sched make_sched(int n_pairs, int I, int grid, int identity) {
     Sched sc;
