@@ -51,7 +51,7 @@ void prof_reset() {
 struct Plan {
     size_t status, ids, w, omit_src, omit_tgt, block_hist, sb_hist, offsets, work_start, totals, perm, row_tok, row_w,
         row_exp, pool_ids, pool_size, pool_mask, target, scale, grp_expert, grp_off, n_groups, zeros, calib, big,
-        xs, H, y32, out, grp_tiles, obuf, inv_pos, calib_nrm, calib_warn, w64, total;
+        xs, H, out, grp_tiles, obuf, inv_pos, calib_nrm, calib_warn, w64, total;
 };
 
 bool valid_layer(const exfold_layer* l) {
@@ -117,8 +117,7 @@ Plan make_plan(const exfold_layer& l, int64_t Tm, int Kr) {
         // fp32 per-row expert outputs once GEMM-1 has consumed the gathered rows
         p.xs = p.big;
         a = align_up(Rtot * (size_t)l.hidden * 2, 1024);
-        p.y32 = p.big + a;  // decode: fp32 accumulator [B][d]; prefill: per-route bf16 outputs O [Rtot][d]
-        p.obuf = p.y32;
+        p.obuf = p.big + a;  // per-row bf16 outputs O [Rtot][d] (decode: one plane per K part)
         a += align_up(std::max((size_t)Tm * l.hidden * 4, Rtot * (size_t)l.hidden * 2), 1024);
         p.H = p.big + a;
         a += align_up(Rtot * (size_t)l.inter * 2, 1024);
@@ -466,7 +465,7 @@ int exfold_moe_prefill_ex(const exfold_layer* layer, const void* x, const float*
         g.d = d; g.I = I; g.n_ntiles = (I + 127) / 128; g.ksplit = 1; g.a_rows = kTileM;
         g.grp_expert = nullptr; g.n_groups_dev = nullptr;
         g.H = at<__nv_bfloat16>(ws, pl.H); g.row_tok = cp.row_tok; g.row_w = cp.row_w;
-        g.y32 = nullptr; g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
+        g.y = nullptr; g.status = at<DeviceStatus>(ws, pl.status);
         const int64_t max_tiles = Rtot / kTileM + G;
         const int nt1 = (I + 127) / 128, nt2 = (d + 255) / 256;
         GroupedGemmParams g2 = g;  // GEMM-2: H x W_down -> y (or the per-route buffer O)
@@ -647,7 +646,7 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
         g.R = max_rows; g.d = d; g.I = I; g.n_ntiles = (d + 255) / 256; g.ksplit = 1; g.a_rows = a_rows;
         g.grp_expert = rp.grp_expert; g.n_groups_dev = rp.n_groups;
         g.H = fp.H; g.row_tok = rp.row_tok; g.row_w = rp.row_w;
-        g.y32 = nullptr; g.y = at<__nv_bfloat16>(ws, pl.obuf); g.store_rows = 1; g.status = rp.status;
+        g.y = at<__nv_bfloat16>(ws, pl.obuf); g.store_rows = 1; g.status = rp.status;
         // Fewer (expert, column tile) items than half the SMs (few experts, large I): K is split in two so that
         // enough SMs stream W_down; each part's rows go to a plane of their own (the two planes are the row buffer
         // and the unused gathered-rows region before it) and are summed, in order, by the kernel after.

@@ -358,7 +358,7 @@ struct GroupedGemmParams {
     int R;                      // routed rows (shared rows start here)
     int d, I;
     int n_ntiles;               // column tiles
-    int ksplit;                 // GEMM-2: K parts per tile (> 1 only with the y32 reduction epilogue)
+    int ksplit;                 // GEMM-2, decode: K parts per tile; part k of a row goes to plane k of the row buffer
     int a_rows;                 // decode: rows of the A (token) box, a multiple of 32 <= 128; prefill: 128
     const int32_t* grp_expert;  // [G] expert whose weights group g uses (null: g itself)
     const int32_t* n_groups_dev;  // device-side group count (null: G)
@@ -366,7 +366,6 @@ struct GroupedGemmParams {
     __nv_bfloat16* H;           // GEMM-1 out [Rtot][I]
     const int32_t* row_tok;     // GEMM-2
     const float* row_w;         // GEMM-2
-    float* y32;                 // GEMM-2 accumulate target (null: bf16 store into y)
     __nv_bfloat16* y;           // GEMM-2 bf16 target: row = token (store_rows == 0) or the sorted row itself
     int store_rows;             // 1: y is the per-route buffer O[row][d] that the combine kernel sums
     float* o32;                 // GEMM-2, calibration: unweighted fp32 outputs O32[row][d] (null: the epilogues above)
@@ -383,7 +382,7 @@ struct GroupedGemmParams {
 cudaError_t launch_grouped_gemm1(const GroupedGemmParams& p, int grid, cudaStream_t s);
 cudaError_t launch_grouped_gemm2(const GroupedGemmParams& p, int grid, cudaStream_t s);
 // Prefill on CTA pairs: every group's row tiles two at a time (a last odd tile is left to the kernels above with
-// odd_only = 1). GEMM-2 needs tm_b1 = W_down with 128-row boxes. No grp_expert, no K split, y32 = null, o32 = null.
+// odd_only = 1). GEMM-2 needs tm_b1 = W_down with 128-row boxes. No grp_expert, no K split, o32 = null.
 cudaError_t launch_grouped_gemm1_pair(const GroupedGemmParams& p, int grid, cudaStream_t s);
 cudaError_t launch_grouped_gemm2_pair(const GroupedGemmParams& p, int grid, cudaStream_t s);
 // The odd-tile pass beside them (p.odd_only = 1; prefill instantiation), launched two CTAs at a time so that the two

@@ -393,13 +393,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                                 for (int j = 0; j < 32; ++j)
                                     if (col0 + j < p.d) dstf[j] = __uint_as_float(v[j]);
                             }
-                        } else if (p.y32 != nullptr) {
-                            float* dst = p.y32 + (int64_t)tok * p.d + col0;
-#pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                ptx::red_add_v4(dst + 4 * j, wv * __uint_as_float(v[4 * j]),
-                                                wv * __uint_as_float(v[4 * j + 1]), wv * __uint_as_float(v[4 * j + 2]),
-                                                wv * __uint_as_float(v[4 * j + 3]));
                         } else {
                             uint32_t pk[16];
 #pragma unroll
