@@ -263,15 +263,21 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
         for (int w = w_begin; w < total; w += w_stride, ++iter) {
             const int as = iter & 1, aphase = (iter >> 1) & 1;
             const PairItem it = decode_pair(w, G, nt, s_off, s_wp);
+            const int rows = rank ? it.rows1 : kTileM;
+            const int row = q * 32 + lane;
+            const bool valid = row < rows;
+            const int64_t grow = (int64_t)it.row0 + rank * kTileM + row;
+            int tok = 0;  // GEMM-2: the row's token and weight, asked for before the wait for the accumulator
+            float wv = 0.f;
+            if (MODE == 1 && valid) {
+                tok = p.row_tok[grow];
+                wv = p.row_w[grow];
+            }
             int ok = 1;
             if (lane == 0) ok = ptx::mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status, 4) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             ptx::tc_fence_after();
-            const int rows = rank ? it.rows1 : kTileM;
-            const int row = q * 32 + lane;
-            const bool valid = row < rows;
-            const int64_t grow = (int64_t)it.row0 + rank * kTileM + row;
             const uint32_t taddr = tmem_base + as * 256 + ((uint32_t)(q * 32) << 16);
             if (MODE == 0) {
 #pragma unroll 1
@@ -298,12 +304,6 @@ __global__ void __launch_bounds__(kPThreads, 1) grouped_gemm_pair_kernel(const _
                     }
                 }
             } else {
-                int tok = 0;
-                float wv = 0.f;
-                if (valid) {
-                    tok = p.row_tok[grow];
-                    wv = p.row_w[grow];
-                }
 #pragma unroll 1
                 for (int c = 0; c < 8; ++c) {
                     uint32_t v[32];

@@ -130,16 +130,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
     }
     grid_dep_wait();  // everything below reads what the routing kernels (or GEMM-1) wrote
     int G = p.G;
-    if (DEC) {  // the number of groups (pool size) is known only on the device
-        const int gd = *p.n_groups_dev;
-        G = gd < G ? gd : G;
-    }
+    // DEC: the number of groups (pool size) is known only on the device; the tables are read up to the host's upper
+    // bound in the same round trip (rows past the device's count are never used)
+    const int gd = DEC ? *p.n_groups_dev : G;
     for (int i = threadIdx.x; i <= G; i += kGemmThreads) {
         // offsets == null: one group of p.R rows (a plain GEMM, e.g. the router scores)
         s_off[i] = p.offsets != nullptr ? p.offsets[i] : i * p.R;
         s_ws[i] = p.offsets != nullptr ? p.work_start[i] : i * ((p.R + kTileM - 1) / kTileM);
         if (DEC) s_exp[i] = i < G ? p.grp_expert[i] : i;  // group -> expert whose weights it uses
     }
+    if (DEC) G = gd < G ? gd : G;
     ptx::tc_fence_before();
     __syncthreads();
     if (!DEC && p.odd_only) {
@@ -329,6 +329,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
         for (int w = w_begin; w < total; w += w_stride, ++iter) {
             const int as = iter & 1, aphase = (iter >> 1) & 1;
             const WorkItem it = decode_work(w, G, nt, ks, s_off, s_ws, DEC ? 0 : p.odd_only);
+            const int row = q * 32 + lane;
+            const bool valid = row < it.rows && it.kpart * kb_per < nkb;  // a K part without k-blocks adds nothing
+            const int64_t grow = (int64_t)it.row0 + row;
+            int tok = 0;  // GEMM-2: the row's token and weight, asked for before the wait for the accumulator
+            float wv = 0.f;
+            if (MODE == 1 && valid) {
+                tok = p.row_tok[grow];
+                wv = p.row_w[grow];
+            }
             // lane 0 waits; the warp takes one decision, so the warp-wide TMEM loads below stay convergent
             int ok = 1;
             if (lane == 0) {
@@ -338,9 +347,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             ptx::tc_fence_after();
-            const int row = q * 32 + lane;
-            const bool valid = row < it.rows && it.kpart * kb_per < nkb;  // a K part without k-blocks adds nothing
-            const int64_t grow = (int64_t)it.row0 + row;
             const uint32_t taddr = tmem_base + as * 256 + ((uint32_t)(q * 32) << 16);
             if (MODE == 0) {
 #pragma unroll 1
@@ -367,12 +373,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) grouped_gemm_kernel(const __g
                     }
                 }
             } else {
-                int tok = 0;
-                float wv = 0.f;
-                if (valid) {
-                    tok = p.row_tok[grow];
-                    wv = p.row_w[grow];
-                }
 #pragma unroll 1
                 for (int c = 0; c < 8; ++c) {
                     uint32_t v[32];
