@@ -609,10 +609,11 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
         int stages = 0, scratch_off = 0, ar = 0;
         decode_ffn_smem_plan((int)B, K, N, &stages, &scratch_off, &ar);
         if (stages < 2) return EXFOLD_ERR_UNSUPPORTED;
-        CUtensorMap tm_x, tm_wg64, tm_wu64;
+        CUtensorMap tm_x, tm_wg64, tm_wu64, tm_wg96, tm_wu96;
         const uint64_t E = (uint64_t)G;
         if (!make_tmap(&tm_x, x, (uint64_t)B, d, ar) || !make_tmap(&tm_wg64, w_gate, E * I, d, 64) ||
-            !make_tmap(&tm_wu64, w_up, E * I, d, 64))
+            !make_tmap(&tm_wu64, w_up, E * I, d, 64) || !make_tmap(&tm_wg96, w_gate, E * I, d, 96) ||
+            !make_tmap(&tm_wu96, w_up, E * I, d, 96))
             return EXFOLD_ERR_CUDA;
         DecodeTopkParams tp{};
         tp.logits = logits; tp.x = reinterpret_cast<const __nv_bfloat16*>(x);
@@ -621,7 +622,7 @@ static int decode_impl(const exfold_layer* layer, const void* x, const float* lo
         tp.ids = rp.ids; tp.w64 = at<double>(ws, pl.w64); tp.status = rp.status;
         { ProfScope ps(6, s); EXFOLD_CUDA(launch_decode_topk(tp, s)); }
         DecodeFfnParams fp{};
-        fp.tm_x = tm_x; fp.tm_wg = tm_wg; fp.tm_wu = tm_wu; fp.tm_wg64 = tm_wg64; fp.tm_wu64 = tm_wu64;
+        fp.tm_x = tm_x; fp.tm_wg = tm_wg; fp.tm_wu = tm_wu; fp.tm_wg64 = tm_wg64; fp.tm_wu64 = tm_wu64; fp.tm_wg96 = tm_wg96; fp.tm_wu96 = tm_wu96;
         fp.ids = rp.ids; fp.w64 = tp.w64; fp.S = tables->S; fp.L = tables->L; fp.h = tables->h;
         fp.st_pool = rp.st_pool; fp.st_target = rp.st_target; fp.st_scale = rp.st_scale;
         fp.B = (int)B; fp.N = N; fp.K = K; fp.M = pool_m; fp.n_shared = l.n_shared; fp.d = d; fp.I = I; fp.a_rows = ar;

@@ -223,6 +223,8 @@ struct DecodeFfnParams {
     CUtensorMap tm_wu;    // W_up
     CUtensorMap tm_wg64;  // the same with 64-row boxes (half-width items)
     CUtensorMap tm_wu64;
+    CUtensorMap tm_wg96;  // and with 96-row boxes (a single round of 96-wide items)
+    CUtensorMap tm_wu96;
     const int32_t* ids;   // [B][K] from the top-k kernel
     const double* w64;    // [B][K]
     const float* S;       // tables (dynamic pool)

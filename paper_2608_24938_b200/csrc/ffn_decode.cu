@@ -70,6 +70,7 @@ struct Item {
 
 struct Sched {  // the same in every role of a CTA
     int n_pairs, nfull, has_half, f_keep, split, total;
+    int n96;       // > 0: every item is a 96-wide slice, n96 per pair (see make_sched)
     int identity;  // pair p is (group p, token tile 0): no list needed
     int ctas;      // CTAs that take work: item w belongs to CTA w % ctas
 };
@@ -90,6 +91,18 @@ __device__ __forceinline__ Sched make_sched(int n_pairs, int I, int grid, int id
     const float c = 110.0f;
     const int q = F / grid, r = F % grid;
     const bool can_split = r > 0 && 2 * r + H <= grid;
+    // Less than one round of full items, too many to halve: 96-wide slices when they divide I and still fit one round.
+    // What an SM streams is bounded by the bytes its ring keeps in flight over the loaded HBM latency (~60 GB/s), so a
+    // single round goes faster on more SMs with smaller items (16 experts x 768: 128 items of 0.75 MB, not 96 of 1 MB).
+    sc.n96 = 0;
+    if (q == 0 && r > 0 && !can_split && H == 0 && I % 96 == 0 && n_pairs * (I / 96) <= grid && I / 96 > sc.nfull) {
+        sc.n96 = I / 96;
+        sc.split = 0;
+        sc.ctas = grid;
+        sc.f_keep = 0;
+        sc.total = n_pairs * sc.n96;
+        return sc;
+    }
     float ta = (float)q * fmaxf(1.0f, (float)grid / c);
     if (can_split) ta += 0.5f * fmaxf(1.0f, (float)(2 * r) / c);
     else if (r > 0) ta += fmaxf(1.0f, (float)r / c);
@@ -111,7 +124,11 @@ __device__ __forceinline__ Sched make_sched(int n_pairs, int I, int grid, int id
 __device__ __forceinline__ Item decode_item(int w, const Sched& sc, const Scratch& s, int N) {
     Item it;
     int pair;
-    if (w < sc.f_keep) {
+    if (sc.n96 > 0) {
+        pair = w / sc.n96;
+        it.j0 = (w - pair * sc.n96) * 96;
+        it.s = 96;
+    } else if (w < sc.f_keep) {
         pair = w / sc.nfull;
         it.j0 = (w - pair * sc.nfull) * 128;
         it.s = 128;
@@ -161,6 +178,8 @@ __global__ void __launch_bounds__(kFThreads, 1) decode_ffn_kernel(const __grid_c
         ptx::prefetch_tmap(&p.tm_x);
         ptx::prefetch_tmap(&p.tm_wg);
         ptx::prefetch_tmap(&p.tm_wu);
+        ptx::prefetch_tmap(&p.tm_wg96);
+        ptx::prefetch_tmap(&p.tm_wu96);
         for (int s = 0; s < kFMaxStages; ++s) {
             ptx::mbar_init(&full_bar[s], 1);
             ptx::mbar_init(&empty_bar[s], 1);
@@ -438,6 +457,9 @@ __global__ void __launch_bounds__(kFThreads, 1) decode_ffn_kernel(const __grid_c
                         if (it.s == 128) {
                             ptx::tma_load_2d(b_dst, &p.tm_wg, &full_bar[stage], kb * kFBK, wrow);
                             ptx::tma_load_2d(b_dst + 128 * kFBK * 2, &p.tm_wu, &full_bar[stage], kb * kFBK, wrow);
+                        } else if (it.s == 96) {
+                            ptx::tma_load_2d(b_dst, &p.tm_wg96, &full_bar[stage], kb * kFBK, wrow);
+                            ptx::tma_load_2d(b_dst + 96 * kFBK * 2, &p.tm_wu96, &full_bar[stage], kb * kFBK, wrow);
                         } else {
                             ptx::tma_load_2d(b_dst, &p.tm_wg64, &full_bar[stage], kb * kFBK, wrow);
                             ptx::tma_load_2d(b_dst + 64 * kFBK * 2, &p.tm_wu64, &full_bar[stage], kb * kFBK, wrow);
@@ -458,7 +480,8 @@ __global__ void __launch_bounds__(kFThreads, 1) decode_ffn_kernel(const __grid_c
             const uint32_t lo0 = (ptx::smem_u32(tiles) & 0x3FFFFu) >> 4;
             const uint32_t lo_step = (uint32_t)stage_bytes >> 4, lo_b = (uint32_t)a_bytes >> 4;
             const uint32_t desc_hi32 = (uint32_t)(ptx::make_kmajor_sw128_desc(0) >> 32);
-            constexpr uint32_t idesc256 = ptx::make_idesc_bf16(128, 256), idesc128 = ptx::make_idesc_bf16(128, 128);
+            constexpr uint32_t idesc256 = ptx::make_idesc_bf16(128, 256), idesc128 = ptx::make_idesc_bf16(128, 128),
+                               idesc192 = ptx::make_idesc_bf16(128, 192);
             int stage = 0, phase = 0, item = 0;
             uint32_t a_lo = lo0;
             bool ok = true, ready = false;
@@ -468,7 +491,7 @@ __global__ void __launch_bounds__(kFThreads, 1) decode_ffn_kernel(const __grid_c
                 if (!ptx::mbar_wait(&tempty_bar[as], aphase ^ 1, abort_flag, p.status, 2)) break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + as * 256;
-                const uint32_t idesc = it.s == 128 ? idesc256 : idesc128;
+                const uint32_t idesc = it.s == 128 ? idesc256 : (it.s == 96 ? idesc192 : idesc128);
                 for (int kb = 0; kb < nkb; ++kb) {
                     if (!ready && !ptx::mbar_wait(&full_bar[stage], phase, abort_flag, p.status, 3)) {
                         ok = false;
