@@ -280,3 +280,20 @@ def test_shared_expert_pairs_under_graph_capture():
     assert np.array_equal(got, ref)
     idx = sample_tokens(T, 40)
     check_output(got[idx], case.oracle_prefill(Kp, tok_idx=idx)["y"], "bf16")
+
+
+# ------------------------------------------------------------------ decode work lists: every slicing of the gate/up kernel
+@pytest.mark.parametrize("N,K,B,M,inter", [
+    (64, 4, 64, 30, 384),    # 30 x 3 full slices < one round, too many to halve, 96 | I: 96-wide slices (120 items)
+    (64, 4, 64, 20, 384),    # 60 full slices: the whole round is cut into halves
+    (64, 4, 64, 30, 448),    # I = 3 x 128 + 64: full slices plus a natural half per expert
+    (128, 8, 128, 64, 384),  # more than one round: full slices, the last partial round in halves
+])
+def test_decode_slicing_variants(N, K, B, M, inter):
+    """The gate/up kernel deals (pool expert, slice of I) items over the SMs in several ways depending on how many there
+    are (full 128-wide slices, halves, 96-wide slices, a fixed number of CTAs): each against the oracle, with the pool
+    and the remapped slots bit-exact."""
+    case = Case(small_bf16(n_experts=N, top_k=K, decode_batch=B, inter=inter, hidden=256, logits="normal"), std=0.1)
+    got, ref = case.run_decode(M), case.oracle_decode(M)
+    check_decode_meta(got, ref, M)
+    check_output(got["y"], ref["y"], "bf16")
