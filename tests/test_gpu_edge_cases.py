@@ -297,3 +297,23 @@ def test_decode_slicing_variants(N, K, B, M, inter):
     got, ref = case.run_decode(M), case.oracle_decode(M)
     check_decode_meta(got, ref, M)
     check_output(got["y"], ref["y"], "bf16")
+
+
+def test_chunked_host_prefill_with_a_shared_expert():
+    """A host-buffer prefill call long enough to run in chunks, on a layer with a shared expert: every chunk forks
+    the second stream twice (the shared expert's gate/up pairs beside the scatter kernel, then the odd-tile passes)
+    while the copy streams bring the next chunk in and the previous one out. Same bits as the call on device buffers."""
+    cfg = small_bf16(prefill_tokens=8500, n_experts=8, n_shared=1, hidden=128, inter=128, top_k=2, logits="normal")
+    case = Case(cfg)
+    ex, T, K, Kp = case.ex, case.T, cfg.top_k, 1
+    ref = case.run_prefill(Kp, with_meta=False)["y"]
+    ws = ex.alloc_workspace(case.layer, T, K, host_staging=True)
+    ws.fill_(0xFF)
+    xh, lh = case.x.pin_memory(), case.lg.pin_memory()
+    for _ in range(2):
+        yh = torch.full((T, cfg.hidden), float("nan"), dtype=torch.bfloat16).pin_memory()
+        ex.exfold_moe_prefill_host(case.layer, xh, lh, case.d_wg, case.d_wu, case.d_wd, case.tables, Kp, yh, ws)
+        assert ex.exfold_device_status(ws) == 0
+        assert np.array_equal(yh.float().numpy(), ref)
+    idx = sample_tokens(T, 40)
+    check_output(ref[idx], case.oracle_prefill(Kp, tok_idx=idx)["y"], "bf16")
